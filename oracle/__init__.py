@@ -1,0 +1,18 @@
+"""CPU oracle (test infrastructure, not the product).
+
+Plain fp64 restatement of the blockwise verification step, written from the
+paper's definitions in ``tsd_oracle.c`` and loaded here through ctypes.  Only
+tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library never does, and the two share no code.
+
+``theorem1`` holds the toy-model harness for the exactness theorem.
+"""
+from .binding import (  # noqa: F401
+    build,
+    num_threads,
+    dense_mask,
+    masked_attention,
+    confidence_topk,
+    decode_rule,
+    accept,
+)

@@ -1,0 +1,137 @@
+"""ctypes binding of the C oracle: argument marshalling only (numpy arrays in,
+numpy arrays out).  The arithmetic lives in ``tsd_oracle.c``."""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tsd_oracle.c")
+_LIB = os.path.join(_HERE, "libtsd_oracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (-O2, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", _SRC, "-o", tmp, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_num_threads.restype = ctypes.c_int
+        _lib.oracle_decode_rule.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads():
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _arr(x, dtype):
+    if x is None:
+        return None
+    if hasattr(x, "detach"):  # torch tensor
+        x = x.detach().cpu()
+        if str(x.dtype) == "torch.bfloat16":
+            x = x.float()
+        x = x.numpy()
+    return np.ascontiguousarray(x, dtype=dtype)
+
+
+def dense_mask(S, B, R, Nc, vis=None, cache_lens=None):
+    """uint8 [S, B*R, Nc+B*R], 1 = visible (Section 3.3)."""
+    vis = _arr(vis, np.uint64)
+    cache_lens = _arr(cache_lens, np.int32)
+    out = np.empty((S, B * R, Nc + B * R), dtype=np.uint8)
+    _load().oracle_dense_mask(S, B, R, Nc, _ptr(vis), _ptr(cache_lens), _ptr(out))
+    return out
+
+
+def masked_attention(q, k_cache, v_cache, k_draft, v_draft, mask, sm_scale):
+    """q [S,N,Hq,d], k/v_cache [S,Nc,Hkv,d], k/v_draft [S,N,Hkv,d], mask
+    [S,N,Nc+N] -> (out fp64 [S,N,Hq,d], lse fp64 [S,Hq,N])."""
+    q = _arr(q, np.float32)
+    kc, vc = _arr(k_cache, np.float32), _arr(v_cache, np.float32)
+    kd, vd = _arr(k_draft, np.float32), _arr(v_draft, np.float32)
+    mask = _arr(mask, np.uint8)
+    S, N, Hq, d = q.shape
+    Nc, Hkv = kc.shape[1], kc.shape[2]
+    assert kc.shape == (S, Nc, Hkv, d) and vc.shape == kc.shape
+    assert kd.shape == (S, N, Hkv, d) and vd.shape == kd.shape
+    assert mask.shape == (S, N, Nc + N) and Hq % Hkv == 0
+    out = np.empty((S, N, Hq, d), dtype=np.float64)
+    lse = np.empty((S, Hq, N), dtype=np.float64)
+    _load().oracle_masked_attention(
+        S, N, Nc, Hq, Hkv, d, _ptr(q), _ptr(kc), _ptr(vc), _ptr(kd), _ptr(vd),
+        _ptr(mask), ctypes.c_double(float(sm_scale)), _ptr(out), _ptr(lse))
+    return out, lse
+
+
+def confidence_topk(logits, k):
+    """logits [rows, V] -> conf fp64 [rows], idx int32 [rows,k], prob fp64
+    [rows,k], lse fp64 [rows] (Eq. 2; order: logit desc, index asc)."""
+    logits = _arr(logits, np.float32)
+    rows, V = logits.shape
+    assert 1 <= k <= V
+    conf = np.empty(rows, dtype=np.float64)
+    idx = np.empty((rows, k), dtype=np.int32)
+    prob = np.empty((rows, k), dtype=np.float64)
+    lse = np.empty(rows, dtype=np.float64)
+    _load().oracle_confidence_topk(
+        _ptr(logits), ctypes.c_int64(rows), V, ctypes.c_int64(V), k,
+        _ptr(conf), _ptr(idx), _ptr(prob), _ptr(lse))
+    return conf, idx, prob, lse
+
+
+def decode_rule(state, mask_id, conf, top1, tau):
+    """One node: (flag uint8 [R], tok int32 [R]) = U(node)."""
+    state = _arr(state, np.int32)
+    conf = _arr(conf, np.float32)
+    top1 = _arr(top1, np.int32)
+    R = state.shape[0]
+    flag = np.empty(R, dtype=np.uint8)
+    tok = np.empty(R, dtype=np.int32)
+    _load().oracle_decode_rule(R, _ptr(state), ctypes.c_int32(mask_id), _ptr(conf),
+                               _ptr(top1), ctypes.c_float(tau), _ptr(flag), _ptr(tok))
+    return flag, tok
+
+
+def accept(parent, state, mask_id, conf, top1, tau, rule=0, search=0):
+    """parent [S,B], state [S,B,R], conf [S,B,R] fp32, top1 [S,B,R] ->
+    dict of edge_valid, prefix_len, accepted_node, accepted_len,
+    n_new_tokens, unmask_flag, unmask_tok."""
+    parent = _arr(parent, np.int32)
+    state = _arr(state, np.int32)
+    conf = _arr(conf, np.float32)
+    top1 = _arr(top1, np.int32)
+    S, B, R = state.shape
+    assert parent.shape == (S, B) and conf.shape == (S, B, R) and top1.shape == (S, B, R)
+    o = dict(
+        edge_valid=np.empty((S, B), np.uint8),
+        prefix_len=np.empty((S, B), np.int32),
+        accepted_node=np.empty(S, np.int32),
+        accepted_len=np.empty(S, np.int32),
+        n_new_tokens=np.empty(S, np.int32),
+        unmask_flag=np.empty((S, R), np.uint8),
+        unmask_tok=np.empty((S, R), np.int32),
+    )
+    _load().oracle_accept(
+        S, B, R, _ptr(parent), _ptr(state), ctypes.c_int32(mask_id), _ptr(conf),
+        _ptr(top1), ctypes.c_int64(1), ctypes.c_float(tau), int(rule), int(search),
+        _ptr(o["edge_valid"]), _ptr(o["prefix_len"]), _ptr(o["accepted_node"]),
+        _ptr(o["accepted_len"]), _ptr(o["n_new_tokens"]), _ptr(o["unmask_flag"]),
+        _ptr(o["unmask_tok"]))
+    return o

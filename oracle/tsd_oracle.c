@@ -1,0 +1,325 @@
+/*
+ * CPU oracle for the blockwise verification step of trajectory-level
+ * speculative decoding for diffusion language models.
+ *
+ * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a plain, slow,
+ * fp64 restatement of what the verification step computes, written from the
+ * paper's definitions.  It shares no code with the CUDA library; only tests,
+ * the smoke check and the benchmark's CPU-baseline leg may call it.
+ *
+ * Inputs that the GPU receives as bf16 or fp32 arrive here as fp32 arrays
+ * (both widen to fp32 exactly); all arithmetic below is in double.
+ *
+ * Parts, and the passage each follows:
+ *   oracle_dense_mask        Section 3.3, the two visibility rules + "bidirectional"
+ *   oracle_masked_attention  Section 3.3 / App. A: softmax attention under that mask
+ *   oracle_confidence_topk   Eq. 2 (confidence) and the top-k candidates of Section 3.2
+ *   oracle_decode_rule       Alg. 1 Phase 1 (H = {conf > tau}) with the top-1
+ *                            fallback of Eqs. 6-7
+ *   oracle_accept            Section 3.3 "Verification procedure" (greedy / longest path)
+ *
+ * Pins (tests/test_oracle_*.py): textbook attention for one branch, plain
+ * bidirectional attention for an all-visible mask, per-row brute force,
+ * closed forms, hand-worked acceptance trees, and the exactness theorem
+ * (Theorem 1) on a toy model.  The paper prints no numeric value for this
+ * path, so parity against printed values is unpinned; parity is against the
+ * definitions and invariants listed above.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------
+ * Section 3.3.  Keys are laid out as [cached prefix+suffix tokens | draft rows
+ * of branch 0 | draft rows of branch 1 | ...].  Query row i belongs to branch
+ * b = i / R.  Rule 1: every row of a draft block sees all cached tokens
+ * (those below cache_lens[s] when a sequence holds fewer than Nc).  Rule 2:
+ * it sees no row of another draft block.  "Bidirectional" inside the block:
+ * it sees every row of its own block, itself included.  A caller-supplied
+ * bitset vis[s][b] (bit j = branch b may read branch j) generalises rule 2;
+ * the own-branch bit is always taken as set.
+ * ---------------------------------------------------------------------- */
+void oracle_dense_mask(int S, int B, int R, int Nc, const uint64_t* vis,
+                       const int32_t* cache_lens, uint8_t* mask) {
+  const int N = B * R;
+  const int W = (B + 63) / 64;
+  const int64_t L = (int64_t)Nc + N;
+  for (int s = 0; s < S; ++s) {
+    const int clen = cache_lens ? cache_lens[s] : Nc;
+    for (int i = 0; i < N; ++i) {
+      uint8_t* row = mask + ((int64_t)s * N + i) * L;
+      const int b = i / R;
+      for (int j = 0; j < Nc; ++j) row[j] = (uint8_t)(j < clen);
+      for (int j = 0; j < N; ++j) {
+        const int bj = j / R;
+        int visible = (bj == b);
+        if (vis && !visible) {
+          const uint64_t w = vis[((int64_t)s * B + b) * W + bj / 64];
+          visible = (int)((w >> (bj % 64)) & 1u);
+        }
+        row[Nc + j] = (uint8_t)visible;
+      }
+    }
+  }
+}
+
+/* ------------------------------------------------------------------------
+ * Masked softmax attention, one (sequence, head, draft row) at a time.
+ *   a_j  = sm_scale * <q_i, k_j>        for visible j
+ *   O_i  = sum_j exp(a_j - max a) v_j / sum_j exp(a_j - max a)
+ *   lse  = max a + log sum_j exp(a_j - max a)
+ * Grouped-query heads: query head h reads kv head h / (Hq / Hkv).
+ * Layouts (contiguous): q,out [S,N,Hq,d]; kc,vc [S,Nc,Hkv,d]; kd,vd [S,N,Hkv,d];
+ * mask [S,N,Nc+N]; lse [S,Hq,N] (nullable).
+ * ---------------------------------------------------------------------- */
+void oracle_masked_attention(int S, int N, int Nc, int Hq, int Hkv, int d,
+                             const float* q, const float* kc, const float* vc,
+                             const float* kd, const float* vd,
+                             const uint8_t* mask, double sm_scale, double* out,
+                             double* lse) {
+  const int64_t L = (int64_t)Nc + N;
+  const int group = Hq / Hkv;
+  const int64_t total = (int64_t)S * Hq * N;
+#pragma omp parallel
+  {
+    double* a = (double*)malloc(sizeof(double) * (size_t)L);
+    double* acc = (double*)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 8)
+    for (int64_t t = 0; t < total; ++t) {
+      const int i = (int)(t % N);
+      const int h = (int)((t / N) % Hq);
+      const int s = (int)(t / ((int64_t)N * Hq));
+      const int g = h / group;
+      const uint8_t* mrow = mask + ((int64_t)s * N + i) * L;
+      const float* qi = q + (((int64_t)s * N + i) * Hq + h) * d;
+      double amax = -INFINITY;
+      for (int64_t j = 0; j < L; ++j) {
+        if (!mrow[j]) continue;
+        const float* kj = (j < Nc)
+                              ? kc + (((int64_t)s * Nc + j) * Hkv + g) * d
+                              : kd + (((int64_t)s * N + (j - Nc)) * Hkv + g) * d;
+        double dot = 0.0;
+        for (int c = 0; c < d; ++c) dot += (double)qi[c] * (double)kj[c];
+        a[j] = sm_scale * dot;
+        if (a[j] > amax) amax = a[j];
+      }
+      double z = 0.0;
+      for (int c = 0; c < d; ++c) acc[c] = 0.0;
+      for (int64_t j = 0; j < L; ++j) {
+        if (!mrow[j]) continue;
+        const float* vj = (j < Nc)
+                              ? vc + (((int64_t)s * Nc + j) * Hkv + g) * d
+                              : vd + (((int64_t)s * N + (j - Nc)) * Hkv + g) * d;
+        const double p = exp(a[j] - amax);
+        z += p;
+        for (int c = 0; c < d; ++c) acc[c] += p * (double)vj[c];
+      }
+      double* oi = out + (((int64_t)s * N + i) * Hq + h) * d;
+      for (int c = 0; c < d; ++c) oi[c] = acc[c] / z;
+      if (lse) lse[((int64_t)s * Hq + h) * N + i] = amax + log(z);
+    }
+    free(a);
+    free(acc);
+  }
+}
+
+/* ------------------------------------------------------------------------
+ * Eq. 2 and the candidate pool of Section 3.2.  Per row of logits l[0..V):
+ *   m = max l,  Z = sum exp(l - m),  p_v = exp(l_v - m) / Z,
+ *   conf = max_v p_v = p of the first candidate,
+ *   candidates = the first k vocabulary entries in the order
+ *                (logit descending, index ascending),
+ *   lse = m + log Z.
+ * The order is decided on the raw input values, so the indices are unique.
+ * Selection is k plain scans: scan t picks the best entry that comes
+ * strictly after the previous pick in that order.
+ * ---------------------------------------------------------------------- */
+static int comes_before(float va, int ia, float vb, int ib) {
+  /* 1 if (va, ia) precedes (vb, ib): larger logit first, then lower index */
+  if (va > vb) return 1;
+  if (va < vb) return 0;
+  return ia < ib;
+}
+
+void oracle_confidence_topk(const float* logits, int64_t n_rows, int V,
+                            int64_t row_stride, int k, double* conf,
+                            int32_t* topk_idx, double* topk_prob, double* lse) {
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t r = 0; r < n_rows; ++r) {
+    const float* l = logits + r * row_stride;
+    double m = -INFINITY;
+    for (int v = 0; v < V; ++v)
+      if ((double)l[v] > m) m = (double)l[v];
+    double z = 0.0;
+    for (int v = 0; v < V; ++v) z += exp((double)l[v] - m);
+    int have_prev = 0, prev_i = -1;
+    float prev_v = 0.0f;
+    for (int t = 0; t < k; ++t) {
+      int best = -1;
+      for (int v = 0; v < V; ++v) {
+        if (have_prev && !comes_before(prev_v, prev_i, l[v], v)) continue;
+        if (best < 0 || comes_before(l[v], v, l[best], best)) best = v;
+      }
+      topk_idx[r * k + t] = best;
+      topk_prob[r * k + t] = exp((double)l[best] - m) / z;
+      have_prev = 1;
+      prev_v = l[best];
+      prev_i = best;
+    }
+    conf[r] = topk_prob[r * k]; /* Eq. 2: the probability of the first candidate */
+    if (lse) lse[r] = m + log(z);
+  }
+}
+
+/* ------------------------------------------------------------------------
+ * Decode rule U(p) for one node (block state of R rows): what threshold
+ * ("sequential confidence") decoding would unmask next, given the node's
+ * per-row confidence and top-1 token.
+ *   M = rows still holding mask_id
+ *   H = {r in M : conf[r] > tau}                      (Alg. 1, Phase 1: strict >)
+ *   U = {(r, top1[r]) : r in H}                       if H is not empty
+ *   U = {(r*, top1[r*])}, r* = argmax_{r in M} conf   otherwise (Eqs. 6-7;
+ *                                                      lowest row on ties)
+ *   U = {}                                            if M is empty
+ * conf is the fp32 value the interface carries.  flag[r] = 1 for rows in U.
+ * Returns |U|.
+ * ---------------------------------------------------------------------- */
+int oracle_decode_rule(int R, const int32_t* state, int32_t mask_id,
+                       const float* conf, const int32_t* top1, float tau,
+                       uint8_t* flag, int32_t* tok) {
+  int n_high = 0, n_masked = 0, best = -1;
+  for (int r = 0; r < R; ++r) {
+    flag[r] = 0;
+    tok[r] = -1;
+  }
+  for (int r = 0; r < R; ++r) {
+    if (state[r] != mask_id) continue;
+    ++n_masked;
+    if (best < 0 || conf[r] > conf[best]) best = r;
+    if (conf[r] > tau) {
+      flag[r] = 1;
+      tok[r] = top1[r];
+      ++n_high;
+    }
+  }
+  if (n_high > 0) return n_high;
+  if (n_masked == 0) return 0;
+  flag[best] = 1;
+  tok[best] = top1[best];
+  return 1;
+}
+
+/* ------------------------------------------------------------------------
+ * Acceptance (Section 3.3, "Verification procedure").
+ * Tree: parent[s][b] (parent[0] = -1, parent[b] < b), node 0 = root.
+ * Edge parent->c carries the delta D(c) = rows the parent had masked and c
+ * has filled, with c's tokens.  c is malformed if it alters a row the parent
+ * had already filled or re-masks one; a malformed or empty delta is invalid.
+ *   rule 0 (EXACT): D(c) == U(parent) as sets of (row, token)
+ *   rule 1 (TOP1) : every (r, t) in D(c) has t == top1[parent][r]
+ * prefix_len[b] = number of leading valid edges on the path root -> b.
+ * search 0 (GREEDY): from the root, move to the lowest-index valid child
+ *                    until there is none.
+ * search 1 (LONGEST): the deepest node whose whole path is valid, lowest
+ *                    index among equals.
+ * Outputs per sequence: accepted node, its depth, tokens it holds beyond the
+ * root, and U(accepted node) for the caller's next root.
+ * ---------------------------------------------------------------------- */
+void oracle_accept(int S, int B, int R, const int32_t* parent,
+                   const int32_t* state, int32_t mask_id, const float* conf,
+                   const int32_t* top1, int64_t top1_stride, float tau,
+                   int rule, int search, uint8_t* edge_valid,
+                   int32_t* prefix_len, int32_t* accepted_node,
+                   int32_t* accepted_len, int32_t* n_new_tokens,
+                   uint8_t* unmask_flag, int32_t* unmask_tok) {
+  uint8_t* uflag = (uint8_t*)malloc((size_t)R);
+  int32_t* utok = (int32_t*)malloc(sizeof(int32_t) * (size_t)R);
+  int32_t* t1 = (int32_t*)malloc(sizeof(int32_t) * (size_t)R);
+  int32_t* depth = (int32_t*)malloc(sizeof(int32_t) * (size_t)B);
+  for (int s = 0; s < S; ++s) {
+    const int32_t* par = parent + (int64_t)s * B;
+    uint8_t* ev = edge_valid + (int64_t)s * B;
+    int32_t* pl = prefix_len + (int64_t)s * B;
+    ev[0] = 1;
+    pl[0] = 0;
+    depth[0] = 0;
+    for (int c = 1; c < B; ++c) {
+      const int p = par[c];
+      const int32_t* sp = state + ((int64_t)s * B + p) * R;
+      const int32_t* sc = state + ((int64_t)s * B + c) * R;
+      const float* cp = conf + ((int64_t)s * B + p) * R;
+      for (int r = 0; r < R; ++r)
+        t1[r] = top1[(((int64_t)s * B + p) * R + r) * top1_stride];
+      oracle_decode_rule(R, sp, mask_id, cp, t1, tau, uflag, utok);
+      int n_delta = 0, malformed = 0, ok = 1;
+      for (int r = 0; r < R; ++r) {
+        const int p_masked = (sp[r] == mask_id);
+        const int c_masked = (sc[r] == mask_id);
+        if (!p_masked) {
+          if (sc[r] != sp[r]) malformed = 1;
+          continue;
+        }
+        if (c_masked) {
+          if (rule == 0 && uflag[r]) ok = 0; /* U has a row the delta lacks */
+          continue;
+        }
+        ++n_delta;
+        if (rule == 0) {
+          if (!uflag[r] || utok[r] != sc[r]) ok = 0;
+        } else {
+          if (t1[r] != sc[r]) ok = 0;
+        }
+      }
+      ev[c] = (uint8_t)(ok && !malformed && n_delta > 0);
+      depth[c] = depth[p] + 1;
+      pl[c] = (pl[p] == depth[p] && ev[c]) ? depth[c] : pl[p];
+    }
+    int acc = 0;
+    if (search == 0) {
+      for (;;) {
+        int next = -1;
+        for (int c = 1; c < B; ++c)
+          if (par[c] == acc && ev[c]) {
+            next = c;
+            break;
+          }
+        if (next < 0) break;
+        acc = next;
+      }
+    } else {
+      for (int b = 1; b < B; ++b)
+        if (pl[b] == depth[b] && depth[b] > depth[acc]) acc = b;
+    }
+    accepted_node[s] = acc;
+    accepted_len[s] = depth[acc];
+    const int32_t* s0 = state + ((int64_t)s * B) * R;
+    const int32_t* sa = state + ((int64_t)s * B + acc) * R;
+    int f0 = 0, fa = 0;
+    for (int r = 0; r < R; ++r) {
+      f0 += (s0[r] != mask_id);
+      fa += (sa[r] != mask_id);
+    }
+    n_new_tokens[s] = fa - f0;
+    for (int r = 0; r < R; ++r)
+      t1[r] = top1[(((int64_t)s * B + acc) * R + r) * top1_stride];
+    oracle_decode_rule(R, sa, mask_id, conf + ((int64_t)s * B + acc) * R, t1,
+                       tau, unmask_flag + (int64_t)s * R,
+                       unmask_tok + (int64_t)s * R);
+  }
+  free(uflag);
+  free(utok);
+  free(t1);
+  free(depth);
+}
