@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the blockwise verification step (attention -> confidence/top-k -> acceptance).
+
+One "step" is one pass of the whole hot path over one synthetic batch shaped like the named
+workload.  Prints ONE JSON line: verified draft-token rows per second (device-resident inputs),
+the same measured end to end from pinned host buffers, the roofline of the dominant kernel, and
+the CPU oracle timed on the host cores beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+N > 1 (under torchrun) runs independent replicas, one per GPU: the path has no exchange step.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "verified draft-token rows/sec (attn+topk+accept)"
+UNIT = "rows/s"
+L2_BYTES = 126 * 1024 * 1024
+ROTATE_BYTES = 640 * 1024 * 1024  # rotate through input copies at least this large in total
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (kernel -> workload -> bytes); None where no capture exists.
+NCU_TRAFFIC = {
+    "confidence_topk": {},
+    "verify_attention": {},
+}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), tflops=float(p["bf16_tflops"]),
+                    tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def algorithmic(cfg):
+    """Bytes and FLOPs the method must move/compute per step (visible keys only)."""
+    es = 4 if cfg.dtype == "f32" else 2
+    rows = cfg.rows
+    attn_flops = 4.0 * rows * (cfg.Nc + cfg.R) * cfg.d * cfg.Hq
+    attn_bytes = es * cfg.d * (2 * cfg.S * cfg.N * cfg.Hq + 2 * cfg.S * cfg.Nc * cfg.Hkv
+                               + 2 * cfg.S * cfg.N * cfg.Hkv)
+    topk_bytes = rows * cfg.V * es + rows * (8 + 8 * cfg.k)
+    return dict(attn_flops=attn_flops, attn_bytes=attn_bytes, topk_bytes=topk_bytes)
+
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out = self.proc.communicate(timeout=5)[0]
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out = self.proc.communicate()[0]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def time_oracle_sample(cfg, attn, vi, budget_s, oracle, np):
+    """Times the oracle on a bounded sample and extrapolates to the full workload.
+
+    Sample: attention for all rows of sequence 0 on the first kv heads (and their query heads),
+    top-k on the first rows, acceptance in full; the head and row counts are chosen from a small
+    calibration run so that the timed part costs about `budget_s` seconds.
+    """
+    S, B, R = cfg.S, cfg.B, cfg.R
+    group = cfg.Hq // cfg.Hkv
+    f32 = lambda t: t.detach().float().cpu().numpy()
+    mask = oracle.dense_mask(1, B, R, cfg.Nc)
+
+    def attn_sample(n_kv):
+        hs = slice(0, n_kv * group)
+        ks = slice(0, n_kv)
+        t0 = time.perf_counter()
+        oracle.masked_attention(f32(attn["q"][0:1, :, hs]), f32(attn["k_cache"][0:1, :, ks]),
+                                f32(attn["v_cache"][0:1, :, ks]), f32(attn["k_draft"][0:1, :, ks]),
+                                f32(attn["v_draft"][0:1, :, ks]), mask, attn["sm_scale"])
+        return time.perf_counter() - t0
+
+    def topk_sample(n_rows):
+        x = f32(vi["logits"][:n_rows])
+        t0 = time.perf_counter()
+        out = oracle.confidence_topk(x, cfg.k)
+        return time.perf_counter() - t0, out
+
+    threads = oracle.num_threads()
+    t_a1 = attn_sample(1)
+    t_k1, _ = topk_sample(min(cfg.rows, 4 * threads))
+    per_head = t_a1
+    per_row = t_k1 / min(cfg.rows, 4 * threads)
+    n_kv = max(1, min(cfg.Hkv, int(0.5 * budget_s / max(per_head, 1e-6))))
+    n_rows = max(1, min(cfg.rows, int(0.5 * budget_s / max(per_row, 1e-9))))
+    t_attn = attn_sample(n_kv)
+    t_topk, (conf, idx, prob, _) = topk_sample(n_rows)
+    # acceptance in full, on confidences of the right shape (values do not change its cost)
+    conf_full = np.resize(conf.astype(np.float32), cfg.rows).reshape(S, B, R)
+    top1_full = np.resize(idx[:, 0], cfg.rows).reshape(S, B, R)
+    t0 = time.perf_counter()
+    oracle.accept(vi["parent"].cpu().numpy(), vi["state"].cpu().numpy(), vi["mask_id"], conf_full,
+                  top1_full, cfg.tau)
+    t_acc = time.perf_counter() - t0
+    t_full = t_attn * (cfg.Hkv / n_kv) * S + t_topk * (cfg.rows / n_rows) + t_acc
+    sample = ("attention: sequence 0, %d of %d kv heads (%d query heads), all %d rows; top-k: first %d of "
+              "%d rows; acceptance: all %d sequences; scaled to the full step"
+              % (n_kv, cfg.Hkv, n_kv * group, cfg.N, n_rows, cfg.rows, S))
+    return dict(value=cfg.rows / t_full, unit=UNIT, cores=threads, kind="oracle", sample=sample,
+                seconds_timed=t_attn + t_topk + t_acc,
+                stage_seconds_full=dict(attention=t_attn * (cfg.Hkv / n_kv) * S,
+                                        topk=t_topk * (cfg.rows / n_rows), accept=t_acc))
+
+
+def run_reference(args, cfg):
+    """The CPU oracle as the reference arm (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2608_27514_b200 import workloads as W
+    oracle.build()
+    attn = W.attention_inputs(cfg, "cpu") if cfg.rows <= 4096 else W.attention_inputs(W.small(cfg, S=1), "cpu")
+    vcfg = cfg if cfg.rows <= 4096 else W.small(cfg, S=1)
+    vi = W.verify_inputs(vcfg, "cpu")
+    if vcfg is not cfg:   # acceptance inputs for the full batch: tile the one generated sequence
+        vi["parent"] = vi["parent"].repeat(cfg.S, 1)
+        vi["state"] = vi["state"].repeat(cfg.S, 1, 1)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    budget = min(budget, 10.0)
+    times, last = [], None
+    for it in range(args.warmup + args.steps):
+        last = time_oracle_sample(cfg, attn, vi, budget, oracle, np)
+        if it >= args.warmup:
+            times.append(cfg.rows / last["value"])
+    ms = 1e3 * sum(times) / len(times)
+    value = cfg.rows / (ms / 1e3)
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=cfg.name, rows=cfg.rows, note="CPU oracle, fp64, sampled and scaled"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle",
+                                  sample=last["sample"]),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="tsd", choices=["tsd", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graph replay")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "tsd" else args.warmup
+
+    from paper_2608_27514_b200 import workloads as W
+    cfg = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2608_27514_b200 import binding as B
+    from paper_2608_27514_b200.step import VerifyStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    B.lib()  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    alg = algorithmic(cfg)
+    pk = peaks()
+    in_bytes = alg["attn_bytes"] + alg["topk_bytes"]
+    n_copies = 1 if in_bytes > 2 * L2_BYTES else int(np.ceil(ROTATE_BYTES / in_bytes))
+    sets = []
+    base_attn = W.attention_inputs(cfg, dev)
+    base_vi = W.verify_inputs(cfg, dev)
+    for c in range(n_copies):
+        clone = lambda t: t.clone() if (c > 0 and torch.is_tensor(t)) else t
+        attn = {k: clone(v) for k, v in base_attn.items()}
+        vi = {k: clone(v) for k, v in base_vi.items() if k != "plan"}
+        step = VerifyStep.for_config(cfg, dev)
+        step.build_mask()
+        sets.append((step, attn, vi))
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def run_step(i):
+        step, attn, vi = sets[i % n_copies]
+        step.run(attn, vi["logits"], vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
+
+    graphs = None
+    use_graph = not args.no_graph
+    if use_graph:
+        # one captured step per input copy; the library calls only enqueue work, so they capture as is
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for i in range(n_copies):
+                run_step(i)
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        graphs = []
+        for i in range(n_copies):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                run_step(i)
+            graphs.append(g)
+
+    def do_step(i):
+        if graphs is not None:
+            graphs[i % n_copies].replay()
+        else:
+            run_step(i)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- timed region A: K whole steps, inputs resident in HBM
+    for i in range(args.warmup):
+        do_step(i)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        do_step(args.warmup + i)
+    e1.record(stream)
+    barrier()
+    elapsed_ms = e0.elapsed_time(e1)
+    for st, _, _ in sets:
+        st.check_status()
+
+    # ---------------- timed region B: each stage alone, back-to-back launches on rotating inputs
+    def time_stage(fn, reps):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(reps):
+            fn(i)
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e-3
+
+    def f_attn(i):
+        step, attn, vi = sets[i % n_copies]
+        step.attention(attn["q"], attn["k_cache"], attn["v_cache"], attn["k_draft"], attn["v_draft"],
+                       attn["sm_scale"])
+
+    def f_topk(i):
+        step, attn, vi = sets[i % n_copies]
+        step.confidence_topk(vi["logits"])
+
+    def f_acc(i):
+        step, attn, vi = sets[i % n_copies]
+        step.accept(vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
+
+    reps = max(args.steps, 20)
+    t_attn, t_topk, t_acc = time_stage(f_attn, reps), time_stage(f_topk, reps), time_stage(f_acc, reps)
+    clocks = sampler.stop()
+
+    # ---------------- end to end: pinned host inputs -> device -> step -> host results
+    step0, attn0, vi0 = sets[0]
+    h_names = ["q", "k_draft", "v_draft"]
+    host = {k: attn0[k].cpu().pin_memory() for k in h_names}
+    host_logits = vi0["logits"].cpu().pin_memory()
+    host_parent, host_state = vi0["parent"].cpu().pin_memory(), vi0["state"].cpu().pin_memory()
+    res_names = ["accepted_node", "accepted_len", "n_new_tokens", "unmask_flag", "unmask_tok"]
+    host_out = {k: torch.empty_like(getattr(step0, k), device="cpu").pin_memory() for k in res_names}
+    h2d = sum(t.numel() * t.element_size() for t in list(host.values()) + [host_logits, host_parent, host_state])
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_step():
+        for k in h_names:
+            attn0[k].copy_(host[k], non_blocking=True)
+        vi0["logits"].copy_(host_logits, non_blocking=True)
+        vi0["parent"].copy_(host_parent, non_blocking=True)
+        vi0["state"].copy_(host_state, non_blocking=True)
+        step0.run(attn0, vi0["logits"], vi0["parent"], vi0["state"], vi0["mask_id"], cfg.tau)
+        for k in res_names:
+            host_out[k].copy_(getattr(step0, k), non_blocking=True)
+        stream.synchronize()   # the caller needs the accepted node before planning the next step
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record(stream)
+    barrier()
+    e2e_ms = max(a.elapsed_time(b), (time.perf_counter() - t0) * 1e3) / e2e_steps
+
+    # ---------------- reduce over ranks (replicas: the slowest rank sets the time)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = elapsed_ms / args.steps
+    value = world * cfg.rows / (ms_per_step * 1e-3)
+
+    # ---------------- roofline of the dominant kernel (+ every stage, for context)
+    attn_flop_time = alg["attn_flops"] / (pk["tflops"] * 1e12)
+    attn_byte_time = alg["attn_bytes"] / (pk["hbm_gbs"] * 1e9)
+    attn_bound = "tensor" if attn_flop_time >= attn_byte_time else "hbm"
+    stages = dict(
+        attention=dict(seconds=t_attn, bound=attn_bound, roofline_seconds=max(attn_flop_time, attn_byte_time),
+                       frac=max(attn_flop_time, attn_byte_time) / t_attn,
+                       tflops=alg["attn_flops"] / t_attn / 1e12, gbs=alg["attn_bytes"] / t_attn / 1e9),
+        topk=dict(seconds=t_topk, bound="hbm", roofline_seconds=alg["topk_bytes"] / (pk["hbm_gbs"] * 1e9),
+                  frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9),
+        accept=dict(seconds=t_acc),
+    )
+    if t_topk >= t_attn:
+        ach = alg["topk_bytes"] / t_topk / 1e9
+        roof = dict(kernel="confidence_topk_kernel", bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC["confidence_topk"].get(cfg.name),
+                    algorithmic_bytes=alg["topk_bytes"], peak_source=pk["source"])
+    elif attn_bound == "tensor":
+        ach = alg["attn_flops"] / t_attn / 1e12
+        roof = dict(kernel="verify_attention", bound="tensor", achieved=ach, peak=pk["tflops"], unit="TFLOP/s",
+                    frac=ach / pk["tflops"], traffic=NCU_TRAFFIC["verify_attention"].get(cfg.name),
+                    algorithmic_flops=alg["attn_flops"], peak_source=pk["source"])
+    else:
+        ach = alg["attn_bytes"] / t_attn / 1e9
+        roof = dict(kernel="verify_attention", bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC["verify_attention"].get(cfg.name),
+                    algorithmic_bytes=alg["attn_bytes"], peak_source=pk["source"])
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cpu = time_oracle_sample(cfg, base_attn, base_vi, 20.0, oracle, np)
+
+    launches_per_step = 3  # attention, confidence/top-k, acceptance (the ticket memset is not a kernel of ours)
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
+        config=dict(workload=cfg.name, batch=cfg.S, branches=cfg.B, rows_per_branch=cfg.R, rows=cfg.rows,
+                    n_cache=cfg.Nc, q_heads=cfg.Hq, kv_heads=cfg.Hkv, head_dim=cfg.d, vocab=cfg.V, k=cfg.k,
+                    tau=cfg.tau, attention_layers_per_step=1, parallelism="replicas" if world > 1 else "1gpu",
+                    l2_hygiene=("inputs larger than L2" if n_copies == 1 else
+                                "rotating %d input copies (%.0f MB total, L2 is 126 MB)"
+                                % (n_copies, n_copies * in_bytes / 1e6)),
+                    launch="cuda graph replay" if graphs is not None else "plain launches"),
+        clocks=clocks,
+        e2e=dict(value=world * cfg.rows / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(h2d),
+                 d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms),
+        gpu_launches=launches_per_step * args.steps,
+        roofline=roof, stages=stages, cpu_baseline=cpu)
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,209 @@
+/*
+ * tsd — blockwise verification for trajectory-level speculative decoding of
+ * diffusion language models, as hand-written sm_100a CUDA kernels behind a
+ * plain C ABI.
+ *
+ * One verification step scores every draft block of a trajectory tree in one
+ * pass (paper Section 3.3): masked attention of each branch's rows over the
+ * shared cached prefix/suffix K/V and over that branch's own rows, then a
+ * per-row vocabulary softmax with confidence and top-k candidates (Eq. 2,
+ * Section 3.2), then the per-branch acceptance test and the tree walk
+ * (Section 3.3, "Verification procedure").
+ *
+ * Conventions for every entry point
+ *   - Returns 0 (TSD_OK) or a negative tsd_error.  Nothing throws.
+ *   - Pointers marked "device" are CUDA device addresses owned by the caller;
+ *     the library never allocates, frees or synchronises, it only enqueues
+ *     work on `stream` (a cudaStream_t; NULL = the default stream).
+ *   - All argument checks run on the host before anything is launched; a
+ *     rejected call launches nothing.  Device arrays cannot be checked on the
+ *     host: a kernel that meets an inconsistent entry (for example a parent
+ *     index out of range) ORs a TSD_STATUS_* bit into `*status` (device,
+ *     nullable) and produces a defined, conservative result instead of
+ *     trapping.  Copy the word back and pass it to tsd_check_status().
+ *   - Results are deterministic: the same inputs give the same bits.
+ *   - Non-finite inputs: -inf logits are ordered last with probability 0;
+ *     NaN anywhere gives unspecified values but never a fault.
+ */
+#ifndef TSD_H_
+#define TSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* tsd_stream_t; /* same type as cudaStream_t */
+
+typedef enum {
+  TSD_OK = 0,
+  TSD_ERR_INVALID_ARG = -1, /* NULL, misaligned, out-of-range or inconsistent argument */
+  TSD_ERR_UNSUPPORTED = -2, /* dtype / head_dim / rows_per_branch outside the supported set */
+  TSD_ERR_WORKSPACE = -3,   /* caller-provided buffer smaller than the *_bytes() query */
+  TSD_ERR_CUDA = -4,        /* a CUDA runtime call failed; see tsd_last_cuda_error() */
+  TSD_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (reported via status) */
+  TSD_ERR_DEVICE_DATA = -6  /* a kernel met inconsistent device data (reported via status) */
+} tsd_error;
+
+typedef enum { TSD_F32 = 0, TSD_BF16 = 1 } tsd_dtype;
+
+/* Which draft blocks count as verified (Section 3.3).  EXACT: the rows and
+ * tokens a child adds equal the set that threshold decoding would unmask at
+ * its parent; this is the test under which Theorem 1 holds.  TOP1: every token
+ * the child adds is its parent's top prediction at that row (the literal
+ * "tokens match the model's top predictions"; admits trajectory drift). */
+typedef enum { TSD_ACCEPT_EXACT = 0, TSD_ACCEPT_TOP1 = 1 } tsd_accept_rule;
+
+/* Greedy search takes the first valid continuation per level; longest-path
+ * search takes the deepest fully valid path (Section 3.3). */
+typedef enum { TSD_SEARCH_GREEDY = 0, TSD_SEARCH_LONGEST = 1 } tsd_search;
+
+/* Bits of the device status word. */
+#define TSD_STATUS_TIMEOUT 0x1u     /* a bounded wait inside a kernel expired      */
+#define TSD_STATUS_BAD_PARENT 0x2u  /* parent[b] outside [0, b) for some b > 0     */
+#define TSD_STATUS_BAD_MASK 0x4u    /* mask blob header does not match the layout  */
+
+/* tsd_verify_attention flags */
+#define TSD_ATTN_FORCE_SIMT 0x1u /* use the CUDA-core kernel even where the tensor-core one applies */
+
+/* Branch / position layout: the paper's prefix P, suffix S and draft blocks
+ * B_i (Section 3.3).  Draft row index inside a sequence = branch * R + r. */
+typedef struct {
+  int32_t batch;           /* independent sequences                                        */
+  int32_t n_branches;      /* tree nodes per sequence, node 0 = root; 1..256               */
+  int32_t rows_per_branch; /* R: 32 (one block), 64 (current + next block) or 128          */
+  int32_t n_cache;         /* cached prefix+suffix tokens per sequence (capacity), >= 0    */
+  int32_t n_q_heads;
+  int32_t n_kv_heads;      /* divides n_q_heads; query head h reads kv head h/(Hq/Hkv)     */
+  int32_t head_dim;        /* 64 or 128                                                    */
+  int32_t dtype;           /* tsd_dtype of Q, K, V and O                                   */
+} tsd_layout;
+
+const char* tsd_strerror(int err);
+/* Text of the last CUDA runtime error seen by this thread's calls ("" if none). */
+const char* tsd_last_cuda_error(void);
+/* Decode a status word copied back from the device: TSD_OK, TSD_ERR_TIMEOUT or
+ * TSD_ERR_DEVICE_DATA. */
+int tsd_check_status(uint32_t status_word);
+
+/* ---------------------------------------------------------------------------
+ * Stage 1a — branch-isolation mask (Section 3.3, "Attention masking for
+ * trajectory isolation"): every row of draft block B_i sees all cached tokens
+ * and, bidirectionally, the rows of B_i itself; it sees no row of another
+ * block B_j.  `vis` generalises the second rule (the inter-block variant of
+ * Section 3.4 lets drafts read the other block's root).
+ *
+ *   vis        device, nullable: uint64 [batch, n_branches, ceil(n_branches/64)];
+ *              bit j of vis[s][b] set = rows of branch b may read the draft keys
+ *              of branch j.  Need not be symmetric.  The own-branch bit is
+ *              always treated as set.  NULL = isolated branches.
+ *   cache_lens device, nullable: int32 [batch], valid cached tokens per sequence
+ *              (clamped to [0, n_cache]); NULL = n_cache everywhere.
+ *   mask_out   device, 16-byte aligned, tsd_branch_mask_bytes() bytes: compact
+ *              per-query-tile visibility lists read by tsd_verify_attention.
+ *              Reusable across layers and steps while layout, vis and
+ *              cache_lens stay the same.
+ *   dense_out  device, nullable: uint8 [batch, B*R, n_cache + B*R], 1 = visible
+ *              (for inspection; the attention kernels do not read it).
+ * ------------------------------------------------------------------------- */
+size_t tsd_branch_mask_bytes(const tsd_layout* layout);
+int tsd_build_branch_mask(const tsd_layout* layout, const uint64_t* vis, const int32_t* cache_lens,
+                          void* mask_out, size_t mask_bytes, uint8_t* dense_out,
+                          tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Stage 1b — verify attention (Section 3.3; App. A: cached prefix/suffix K/V
+ * stay fixed, only block-level K/V change).  For every sequence s, query head
+ * h and draft row i:
+ *     O[i] = sum_j softmax_j(sm_scale * <q_i, k_j>) v_j
+ * over the visible keys j = cached tokens below cache_lens[s] plus the draft
+ * rows of the branches visible to i's branch.  bf16 (or fp32) in, fp32
+ * accumulation, output in the input dtype.
+ *
+ *   mask       device: blob written by tsd_build_branch_mask for the same layout.
+ *   q, out     device: [batch, B*R, n_q_heads, head_dim] addressed through the
+ *              strides (in elements); head_dim contiguous; 16-byte aligned base
+ *              and 16-byte multiples for every stride.
+ *   k_cache, v_cache   device: [batch, n_cache, n_kv_heads, head_dim], shared strides c_*.
+ *   k_draft, v_draft   device: [batch, B*R, n_kv_heads, head_dim], shared strides d_*.
+ *   lse        device, nullable: fp32 [batch, n_q_heads, B*R], natural-log
+ *              sum-exp of the scaled scores.
+ *   sm_scale   usually 1/sqrt(head_dim).
+ *   workspace  device, 16-byte aligned, tsd_verify_attention_workspace_bytes()
+ *              bytes (may be 0, then NULL is accepted).
+ *   flags      TSD_ATTN_* bits.
+ * The tensor-core kernel (tcgen05 MMAs with TMEM accumulators, TMA-staged
+ * tiles) serves bf16 with head_dim 128; other combinations run on CUDA cores.
+ * ------------------------------------------------------------------------- */
+size_t tsd_verify_attention_workspace_bytes(const tsd_layout* layout);
+int tsd_verify_attention(const tsd_layout* layout, const void* mask,
+                         const void* q, int64_t q_stride_b, int64_t q_stride_row, int64_t q_stride_head,
+                         const void* k_cache, const void* v_cache,
+                         int64_t c_stride_b, int64_t c_stride_row, int64_t c_stride_head,
+                         const void* k_draft, const void* v_draft,
+                         int64_t d_stride_b, int64_t d_stride_row, int64_t d_stride_head,
+                         void* out, int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head,
+                         float* lse, float sm_scale, void* workspace, size_t workspace_bytes,
+                         uint32_t flags, uint32_t* status, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Stage 2 — confidence and candidates (Eq. 2: c = max softmax(logits);
+ * Section 3.2: top-k candidates per position).  One streaming pass over the
+ * logits.  Per row: conf = largest softmax probability; topk_idx = the k first
+ * vocabulary entries ordered by (logit descending, index ascending), decided on
+ * the raw input values; topk_prob = their probabilities under the softmax over
+ * the whole vocabulary (not renormalised); lse = log sum exp.
+ *
+ *   logits     device: [n_rows, vocab] of `dtype`, row r at logits + r*row_stride
+ *              elements; base and row_stride*sizeof(elem) 16-byte aligned.
+ *   k          1..8, k <= vocab.
+ *   conf       device fp32 [n_rows];  topk_idx device int32 [n_rows, k];
+ *   topk_prob  device fp32 [n_rows, k];  lse device fp32 [n_rows], nullable.
+ *   workspace  device, 16-byte aligned, tsd_confidence_topk_workspace_bytes()
+ *              bytes: per-segment partial results when a row is split across
+ *              thread blocks (few rows); 0 bytes when it is not.
+ * ------------------------------------------------------------------------- */
+size_t tsd_confidence_topk_workspace_bytes(int64_t n_rows, int32_t vocab, int32_t k);
+int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32_t vocab,
+                        int64_t row_stride, int32_t k, float* conf, int32_t* topk_idx,
+                        float* topk_prob, float* lse, void* workspace, size_t workspace_bytes,
+                        uint32_t* status, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Stage 3 — acceptance (Section 3.3 "Verification procedure"; Alg. 1 Phase 1
+ * for the high/low confidence split; Eqs. 6-7 for the top-1 fallback).
+ * Per node p the decode rule U(p) is what threshold decoding would unmask
+ * next: the masked rows with conf > tau and their top-1 tokens, or, when there
+ * are none, the single masked row of largest conf (lowest row on ties).
+ * Edge parent->c is valid under `rule` (see tsd_accept_rule); a child that
+ * adds nothing, alters a filled row or re-masks one is invalid.
+ *
+ *   parent     device int32 [batch, B]; parent[0] = -1, 0 <= parent[b] < b.
+ *   state      device int32 [batch, B, R]: token id, or mask_id where masked.
+ *   conf       device fp32 [batch, B, R] (stage 2 output).
+ *   top1_idx   device int32, element (s,b,r) at top1_idx[((s*B+b)*R+r)*top1_stride]
+ *              (pass topk_idx with top1_stride = k).
+ *   edge_valid    device uint8 [batch, B]; root = 1.
+ *   prefix_len    device int32 [batch, B]: leading valid edges on the path
+ *                 root -> b (the branch's longest accepted trajectory prefix).
+ *   accepted_node device int32 [batch];  accepted_len device int32 [batch] (its depth).
+ *   n_new_tokens  device int32 [batch]: rows the accepted node holds beyond the root.
+ *   unmask_flag   device uint8 [batch, R], unmask_tok device int32 [batch, R]:
+ *                 U(accepted node), the caller's next root update; tok = -1
+ *                 where flag = 0.
+ * R is 1..128, B is 1..256.
+ * ------------------------------------------------------------------------- */
+int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+                            const int32_t* parent, const int32_t* state, int32_t mask_id,
+                            const float* conf, const int32_t* top1_idx, int32_t top1_stride,
+                            float tau, int32_t rule, int32_t search,
+                            uint8_t* edge_valid, int32_t* prefix_len, int32_t* accepted_node,
+                            int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
+                            int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TSD_H_ */

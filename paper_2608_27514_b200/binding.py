@@ -1,0 +1,182 @@
+"""Thin ctypes binding over the libtsd C ABI: same names, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory; each call extracts
+raw pointers and strides and enqueues the library's kernels on torch's current
+stream (or the one given).  There is no fallback: if the library is missing or
+an argument is rejected, the call raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtsd.so")
+
+TSD_F32, TSD_BF16 = 0, 1
+TSD_ACCEPT_EXACT, TSD_ACCEPT_TOP1 = 0, 1
+TSD_SEARCH_GREEDY, TSD_SEARCH_LONGEST = 0, 1
+TSD_ATTN_FORCE_SIMT = 0x1
+TSD_OK, TSD_ERR_INVALID_ARG, TSD_ERR_UNSUPPORTED, TSD_ERR_WORKSPACE = 0, -1, -2, -3
+TSD_ERR_CUDA, TSD_ERR_TIMEOUT, TSD_ERR_DEVICE_DATA = -4, -5, -6
+
+EXPORTS = (
+    "tsd_strerror", "tsd_last_cuda_error", "tsd_check_status",
+    "tsd_branch_mask_bytes", "tsd_build_branch_mask",
+    "tsd_verify_attention_workspace_bytes", "tsd_verify_attention",
+    "tsd_confidence_topk_workspace_bytes", "tsd_confidence_topk",
+    "tsd_accept_trajectories",
+)
+
+
+class TsdError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = "%s failed: %s (%d)" % (where, strerror(code), code)
+        if code == TSD_ERR_CUDA:
+            msg += ": " + last_cuda_error()
+        super().__init__(msg)
+
+
+class tsd_layout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "batch", "n_branches", "rows_per_branch", "n_cache", "n_q_heads", "n_kv_heads",
+        "head_dim", "dtype")]
+
+
+_lib = None
+_vp, _i32, _i64, _u32, _f32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
+                                     ctypes.c_uint32, ctypes.c_float, ctypes.c_size_t)
+
+
+def lib():
+    """The loaded library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libtsd.so is missing (%s): build it with "
+                               "`python -m paper_2608_27514_b200.build`; there is no fallback" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        L.tsd_strerror.restype = ctypes.c_char_p
+        L.tsd_strerror.argtypes = [ctypes.c_int]
+        L.tsd_last_cuda_error.restype = ctypes.c_char_p
+        L.tsd_check_status.argtypes = [_u32]
+        L.tsd_branch_mask_bytes.restype = _sz
+        L.tsd_branch_mask_bytes.argtypes = [ctypes.POINTER(tsd_layout)]
+        L.tsd_build_branch_mask.argtypes = [ctypes.POINTER(tsd_layout), _vp, _vp, _vp, _sz, _vp, _vp]
+        L.tsd_verify_attention_workspace_bytes.restype = _sz
+        L.tsd_verify_attention_workspace_bytes.argtypes = [ctypes.POINTER(tsd_layout)]
+        L.tsd_verify_attention.argtypes = (
+            [ctypes.POINTER(tsd_layout), _vp] + [_vp, _i64, _i64, _i64] + [_vp, _vp, _i64, _i64, _i64]
+            + [_vp, _vp, _i64, _i64, _i64] + [_vp, _i64, _i64, _i64] + [_vp, _f32, _vp, _sz, _u32, _vp, _vp])
+        L.tsd_confidence_topk_workspace_bytes.restype = _sz
+        L.tsd_confidence_topk_workspace_bytes.argtypes = [_i64, _i32, _i32]
+        L.tsd_confidence_topk.argtypes = [_vp, _i32, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
+                                          _sz, _vp, _vp]
+        L.tsd_accept_trajectories.argtypes = [_i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
+                                              _i32, _i32] + [_vp] * 9
+        _lib = L
+    return _lib
+
+
+def strerror(code):
+    return lib().tsd_strerror(int(code)).decode()
+
+
+def last_cuda_error():
+    return lib().tsd_last_cuda_error().decode()
+
+
+def tsd_check_status(status):
+    """status: int word or a 1-element uint32/int32 tensor (copied back here)."""
+    word = int(status.item()) & 0xFFFFFFFF if hasattr(status, "item") else int(status)
+    return lib().tsd_check_status(word)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(rc, where):
+    if rc != TSD_OK:
+        raise TsdError(rc, where)
+
+
+def dtype_code(dt):
+    if dt == torch.float32:
+        return TSD_F32
+    if dt == torch.bfloat16:
+        return TSD_BF16
+    raise TsdError(TSD_ERR_UNSUPPORTED, "dtype %s" % dt)
+
+
+def make_layout(batch, n_branches, rows_per_branch, n_cache, n_q_heads, n_kv_heads, head_dim, dtype):
+    code = dtype if isinstance(dtype, int) else dtype_code(dtype)
+    return tsd_layout(batch, n_branches, rows_per_branch, n_cache, n_q_heads, n_kv_heads, head_dim, code)
+
+
+def tsd_branch_mask_bytes(layout):
+    return int(lib().tsd_branch_mask_bytes(ctypes.byref(layout)))
+
+
+def tsd_build_branch_mask(layout, vis, cache_lens, mask_out, dense_out=None, stream=None):
+    rc = lib().tsd_build_branch_mask(ctypes.byref(layout), _ptr(vis), _ptr(cache_lens), _ptr(mask_out),
+                                     mask_out.numel() * mask_out.element_size(), _ptr(dense_out),
+                                     _stream(stream))
+    _check(rc, "tsd_build_branch_mask")
+
+
+def tsd_verify_attention_workspace_bytes(layout):
+    return int(lib().tsd_verify_attention_workspace_bytes(ctypes.byref(layout)))
+
+
+def _strides3(t):
+    # [batch, rows, heads, dim] -> (batch, row, head) strides in elements
+    assert t.dim() == 4 and t.stride(3) == 1, "head_dim must be contiguous"
+    return t.stride(0), t.stride(1), t.stride(2)
+
+
+def tsd_verify_attention(layout, mask, q, k_cache, v_cache, k_draft, v_draft, out, lse=None,
+                         sm_scale=1.0, workspace=None, flags=0, status=None, stream=None):
+    assert v_cache is None or v_cache.stride() == k_cache.stride()
+    assert v_draft.stride() == k_draft.stride()
+    cs = _strides3(k_cache) if k_cache is not None else (0, 0, layout.head_dim)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().tsd_verify_attention(
+        ctypes.byref(layout), _ptr(mask), _ptr(q), *_strides3(q), _ptr(k_cache), _ptr(v_cache), *cs,
+        _ptr(k_draft), _ptr(v_draft), *_strides3(k_draft), _ptr(out), *_strides3(out), _ptr(lse),
+        float(sm_scale), _ptr(workspace), ws_bytes, int(flags), _ptr(status), _stream(stream))
+    _check(rc, "tsd_verify_attention")
+
+
+def tsd_confidence_topk_workspace_bytes(n_rows, vocab, k):
+    return int(lib().tsd_confidence_topk_workspace_bytes(int(n_rows), int(vocab), int(k)))
+
+
+def tsd_confidence_topk(logits, k, conf, topk_idx, topk_prob, lse=None, workspace=None, status=None,
+                        stream=None):
+    assert logits.dim() == 2 and logits.stride(1) == 1
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().tsd_confidence_topk(
+        _ptr(logits), dtype_code(logits.dtype), logits.shape[0], logits.shape[1], logits.stride(0),
+        int(k), _ptr(conf), _ptr(topk_idx), _ptr(topk_prob), _ptr(lse), _ptr(workspace), ws_bytes,
+        _ptr(status), _stream(stream))
+    _check(rc, "tsd_confidence_topk")
+
+
+def tsd_accept_trajectories(parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule, search,
+                            edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens,
+                            unmask_flag, unmask_tok, status=None, stream=None):
+    S, B, R = state.shape
+    rc = lib().tsd_accept_trajectories(
+        S, B, R, _ptr(parent), _ptr(state), int(mask_id), _ptr(conf), _ptr(top1_idx), int(top1_stride),
+        float(tau), int(rule), int(search), _ptr(edge_valid), _ptr(prefix_len), _ptr(accepted_node),
+        _ptr(accepted_len), _ptr(n_new_tokens), _ptr(unmask_flag), _ptr(unmask_tok), _ptr(status),
+        _stream(stream))
+    _check(rc, "tsd_accept_trajectories")

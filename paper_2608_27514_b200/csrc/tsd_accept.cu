@@ -1,0 +1,196 @@
+// Stage 3: acceptance of draft trajectories (paper Section 3.3 "Verification procedure";
+// Alg. 1 Phase 1 for the high/low confidence split; Eqs. 6-7 for the top-1 fallback).
+//
+// One thread block per sequence.  Warps take tree nodes in turn: first the decode rule U(p) of
+// every node (what threshold decoding would unmask next), then the validity of every edge, both
+// as warp ballots over the block's rows; one thread then walks the tree (a few dozen nodes).
+// Integer and float compares only: the result is exact.
+#include <limits.h>
+#include <math_constants.h>
+#include "tsd_common.cuh"
+
+namespace tsd {
+
+constexpr int kMaxBranches = 256;
+constexpr int kMaxRows = 128;
+constexpr int kRowWords = kMaxRows / 32;
+constexpr int kAcceptThreads = 256;
+
+__global__ void __launch_bounds__(kAcceptThreads)
+accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
+              int mask_id, const float* __restrict__ conf, const int32_t* __restrict__ top1,
+              int top1_stride, float tau, int rule, int search, uint8_t* __restrict__ edge_valid,
+              int32_t* __restrict__ prefix_len, int32_t* __restrict__ accepted_node,
+              int32_t* __restrict__ accepted_len, int32_t* __restrict__ n_new_tokens,
+              uint8_t* __restrict__ unmask_flag, int32_t* __restrict__ unmask_tok,
+              uint32_t* __restrict__ status) {
+  __shared__ uint32_t s_u[kMaxBranches][kRowWords];  // U(p) as a row bitset
+  __shared__ uint8_t s_valid[kMaxBranches];
+  __shared__ int s_par[kMaxBranches];
+  __shared__ int s_acc;
+  const int s = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  const unsigned full = 0xffffffffu;
+  const int32_t* st = state + (size_t)s * B * R;
+  const float* cf = conf + (size_t)s * B * R;
+  const int32_t* t1 = top1 + (size_t)s * B * R * top1_stride;
+  const int words = (R + 31) / 32;
+
+  // decode rule U(p) for every node
+  for (int p = warp; p < B; p += n_warps) {
+    uint32_t hi[kRowWords], any_hi = 0, any_masked = 0;
+    float best = -CUDART_INF_F;
+    int best_r = INT_MAX;
+#pragma unroll
+    for (int w = 0; w < kRowWords; ++w) {
+      hi[w] = 0;
+      if (w < words) {
+        const int r = w * 32 + lane;
+        bool masked = false, high = false;
+        if (r < R) {
+          masked = st[p * R + r] == mask_id;
+          const float c = cf[p * R + r];
+          high = masked && c > tau;  // strictly above the threshold
+          if (masked && (best_r == INT_MAX || c > best)) { best = c; best_r = r; }  // rows ascend
+        }
+        hi[w] = __ballot_sync(full, high);
+        any_hi |= hi[w];
+        any_masked |= __ballot_sync(full, masked);
+      }
+    }
+    if (!any_hi && any_masked) {  // no row above tau: the single most confident masked row
+#pragma unroll
+      for (int off = 16; off; off >>= 1) {
+        const float ov = __shfl_xor_sync(full, best, off);
+        const int orow = __shfl_xor_sync(full, best_r, off);
+        const bool take = orow != INT_MAX &&
+                          (best_r == INT_MAX || ov > best || (ov == best && orow < best_r));
+        if (take) { best = ov; best_r = orow; }
+      }
+#pragma unroll
+      for (int w = 0; w < kRowWords; ++w) hi[w] = (best_r >> 5) == w ? (1u << (best_r & 31)) : 0u;
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int w = 0; w < kRowWords; ++w) s_u[p][w] = hi[w];
+      int par = p == 0 ? -1 : parent[(size_t)s * B + p];
+      if (p > 0 && (par < 0 || par >= p)) {
+        if (status) atomicOr(status, TSD_STATUS_BAD_PARENT);
+        par = -1;  // treated as an invalid edge hanging off nothing
+      }
+      s_par[p] = par;
+    }
+  }
+  __syncthreads();
+
+  // validity of every edge parent -> c
+  for (int c = warp; c < B; c += n_warps) {
+    const int p = s_par[c];
+    bool ok = true, malformed = false, delta = false;
+    if (c > 0 && p >= 0) {
+      for (int w = 0; w < words; ++w) {
+        const int r = w * 32 + lane;
+        if (r < R) {
+          const int sp = st[p * R + r], sc = st[c * R + r];
+          const bool p_masked = sp == mask_id, c_masked = sc == mask_id;
+          const bool in_u = (s_u[p][w] >> lane) & 1u;
+          if (!p_masked) {
+            malformed |= sc != sp;
+          } else if (c_masked) {
+            if (rule == TSD_ACCEPT_EXACT && in_u) ok = false;  // U has a row the child lacks
+          } else {
+            delta = true;
+            const bool tok_ok = t1[(size_t)(p * R + r) * top1_stride] == sc;
+            if (rule == TSD_ACCEPT_EXACT) ok &= in_u && tok_ok; else ok &= tok_ok;
+          }
+        }
+      }
+    }
+    const bool all_ok = __all_sync(full, ok), any_bad = __any_sync(full, malformed),
+               any_delta = __any_sync(full, delta);
+    if (lane == 0) s_valid[c] = c == 0 ? 1 : (p >= 0 && all_ok && !any_bad && any_delta);
+  }
+  __syncthreads();
+
+  // tree walk (parents precede children, so one ascending sweep fills depth and prefix length)
+  if (threadIdx.x == 0) {
+    // prefix_len is read back from the global array this block has just written; a node's depth
+    // is found by walking its parents (trees are a few levels deep)
+    int32_t* pl = prefix_len + (size_t)s * B;
+    uint8_t* ev = edge_valid + (size_t)s * B;
+    int acc = 0, acc_depth = 0;
+    pl[0] = 0;
+    ev[0] = 1;
+    for (int b = 1; b < B; ++b) {
+      const int p = s_par[b];
+      ev[b] = s_valid[b];
+      int depth_p = 0;
+      for (int a = p; a > 0; a = s_par[a]) ++depth_p;
+      const int plp = p >= 0 ? pl[p] : 0;
+      const bool whole = p >= 0 && plp == depth_p && s_valid[b];
+      pl[b] = whole ? depth_p + 1 : plp;
+      if (search == TSD_SEARCH_LONGEST && whole && depth_p + 1 > acc_depth) { acc = b; acc_depth = depth_p + 1; }
+    }
+    if (search == TSD_SEARCH_GREEDY) {
+      for (;;) {
+        int next = -1;
+        for (int b = acc + 1; b < B; ++b)
+          if (s_par[b] == acc && s_valid[b]) { next = b; break; }
+        if (next < 0) break;
+        acc = next;
+        ++acc_depth;
+      }
+    }
+    accepted_node[s] = acc;
+    accepted_len[s] = acc_depth;
+    s_acc = acc;
+  }
+  __syncthreads();
+
+  // tokens gained and the next unmask set U(accepted node)
+  const int acc = s_acc;
+  if (warp == 0) {
+    int gained = 0;
+    for (int w = 0; w < words; ++w) {
+      const int r = w * 32 + lane;
+      bool f0 = false, fa = false;
+      if (r < R) { f0 = st[r] != mask_id; fa = st[acc * R + r] != mask_id; }
+      gained += __popc(__ballot_sync(full, fa)) - __popc(__ballot_sync(full, f0));
+      if (r < R) {
+        const bool in_u = (s_u[acc][w] >> lane) & 1u;
+        unmask_flag[(size_t)s * R + r] = in_u ? 1 : 0;
+        unmask_tok[(size_t)s * R + r] = in_u ? t1[(size_t)(acc * R + r) * top1_stride] : -1;
+      }
+    }
+    if (lane == 0) n_new_tokens[s] = gained;
+  }
+}
+
+}  // namespace tsd
+
+extern "C" int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+                                       const int32_t* parent, const int32_t* state, int32_t mask_id,
+                                       const float* conf, const int32_t* top1_idx, int32_t top1_stride,
+                                       float tau, int32_t rule, int32_t search, uint8_t* edge_valid,
+                                       int32_t* prefix_len, int32_t* accepted_node,
+                                       int32_t* accepted_len, int32_t* n_new_tokens,
+                                       uint8_t* unmask_flag, int32_t* unmask_tok, uint32_t* status,
+                                       tsd_stream_t stream) {
+  if (batch < 0 || n_branches < 1 || n_branches > tsd::kMaxBranches || rows_per_branch < 1 ||
+      rows_per_branch > tsd::kMaxRows || top1_stride < 1)
+    return TSD_ERR_INVALID_ARG;
+  if (rule != TSD_ACCEPT_EXACT && rule != TSD_ACCEPT_TOP1) return TSD_ERR_INVALID_ARG;
+  if (search != TSD_SEARCH_GREEDY && search != TSD_SEARCH_LONGEST) return TSD_ERR_INVALID_ARG;
+  if (!(tau == tau)) return TSD_ERR_INVALID_ARG;  // NaN threshold
+  if (batch == 0) return TSD_OK;
+  if (!parent || !state || !conf || !top1_idx || !edge_valid || !prefix_len || !accepted_node ||
+      !accepted_len || !n_new_tokens || !unmask_flag || !unmask_tok)
+    return TSD_ERR_INVALID_ARG;
+  tsd::accept_kernel<<<batch, tsd::kAcceptThreads, 0, stream>>>(
+      n_branches, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
+      search, edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
+      unmask_tok, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tsd::cuda_fail(e, "accept_kernel");
+  return TSD_OK;
+}

@@ -149,7 +149,12 @@ def plan_tree(cfg, alpha=(0.85, 0.68)):
             st = state[s, b]
             m_rows = np.flatnonzero(st == mask_id)
             # three distinct planted tokens per row
-            t = np.stack([rng.choice(V - 1, size=3, replace=False) for _ in range(R)])
+            t = rng.integers(0, V - 1, size=(R, 3))
+            while True:
+                dup = (t[:, 0] == t[:, 1]) | (t[:, 0] == t[:, 2]) | (t[:, 1] == t[:, 2])
+                if not dup.any():
+                    break
+                t[dup] = rng.integers(0, V - 1, size=(int(dup.sum()), 3))
             tok[s, b] = t
             no_high = rng.random() < 0.25
             hi = rng.random(R) < cfg.f_high

@@ -1,0 +1,343 @@
+"""GPU parity: every stage of the verification step, called through the C ABI, against the CPU
+oracle on the same seeded inputs.  Integer results (indices, validity, lengths) must be bit-exact;
+attention within 2e-2 abs + 1e-2 rel for bf16 (1e-5 for fp32); probabilities within 1e-5."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from conftest import load_accept_cases
+from paper_2608_27514_b200 import binding as B
+from paper_2608_27514_b200 import workloads as W
+from paper_2608_27514_b200.step import VerifyStep
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+PATHS = [pytest.param(0, id="default"), pytest.param(B.TSD_ATTN_FORCE_SIMT, id="simt")]
+
+
+def _np(t):
+    return t.detach().float().cpu().numpy() if t.dtype == torch.bfloat16 else t.detach().cpu().numpy()
+
+
+def _attn_tol(cfg, ref):
+    if cfg.dtype == "bf16":
+        return 2e-2 + 1e-2 * np.abs(ref)
+    return 1e-5 + 1e-5 * np.abs(ref)
+
+
+def _run_attention(cfg, attn, flags, vis=None, cache_lens=None, want_dense=False):
+    step = VerifyStep.for_config(cfg, DEV)
+    dense = None
+    if want_dense:
+        dense = torch.empty((cfg.S, cfg.N, cfg.Nc + cfg.N), dtype=torch.uint8, device=DEV)
+    step.build_mask(vis, cache_lens, dense)
+    step.attention(attn["q"], attn["k_cache"], attn["v_cache"], attn["k_draft"], attn["v_draft"],
+                   attn["sm_scale"], flags)
+    torch.cuda.synchronize()
+    step.check_status()
+    return step, dense
+
+
+def _check_attention(cfg, attn, flags, vis=None, cache_lens=None, heads=None, seqs=None):
+    """Compare with the oracle; `heads`/`seqs` restrict the oracle to a sample."""
+    step, dense = _run_attention(cfg, attn, flags, vis, cache_lens, want_dense=True)
+    mask = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc,
+                             None if vis is None else vis.cpu().numpy(),
+                             None if cache_lens is None else cache_lens.cpu().numpy())
+    assert np.array_equal(dense.cpu().numpy(), mask)
+    seqs = list(range(cfg.S)) if seqs is None else seqs
+    group = cfg.Hq // cfg.Hkv
+    kv_heads = list(range(cfg.Hkv)) if heads is None else heads
+    worst = 0.0
+    for s in seqs:
+        for g in kv_heads:
+            hs = slice(g * group, (g + 1) * group)
+            sl = lambda t, h: _np(t[s:s + 1][:, :, h])
+            ref, ref_lse = oracle.masked_attention(
+                sl(attn["q"], hs), sl(attn["k_cache"], slice(g, g + 1)), sl(attn["v_cache"], slice(g, g + 1)),
+                sl(attn["k_draft"], slice(g, g + 1)), sl(attn["v_draft"], slice(g, g + 1)),
+                mask[s:s + 1], attn["sm_scale"])
+            got = _np(step.out[s:s + 1][:, :, hs]).astype(np.float64)
+            err = np.abs(got - ref)
+            assert (err <= _attn_tol(cfg, ref)).all(), "attention off by %g (seq %d kv head %d)" % (err.max(), s, g)
+            got_lse = step.attn_lse[s:s + 1, hs].cpu().numpy()
+            assert np.abs(got_lse - ref_lse).max() <= (2e-2 if cfg.dtype == "bf16" else 1e-4)
+            worst = max(worst, err.max())
+    return worst
+
+
+# ----------------------------------------------------------------------------- mask
+def test_mask_dense_matches_oracle_with_vis_and_ragged_cache():
+    cfg = W.small(W.CONFIGS["cfg2"], S=3, B=9, Nc=100, Hq=1, Hkv=1)
+    rng = np.random.default_rng(0)
+    vis = torch.from_numpy(rng.integers(0, 1 << 9, (cfg.S, cfg.B, 1)).astype(np.int64)).to(DEV)
+    lens = torch.tensor([100, 0, 37], dtype=torch.int32, device=DEV)
+    step = VerifyStep.for_config(cfg, DEV)
+    dense = torch.empty((cfg.S, cfg.N, cfg.Nc + cfg.N), dtype=torch.uint8, device=DEV)
+    step.build_mask(vis, lens, dense)
+    torch.cuda.synchronize()
+    ref = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc, vis.cpu().numpy().astype(np.uint64), lens.cpu().numpy())
+    assert np.array_equal(dense.cpu().numpy(), ref)
+
+
+# ------------------------------------------------------------------------ attention
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_cfg1_fp32(flags):
+    cfg = W.CONFIGS["cfg1"]
+    worst = _check_attention(cfg, W.attention_inputs(cfg, DEV), flags)
+    assert worst < 1e-5
+
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("R", [32, 64, 128])
+def test_attention_small_bf16_ragged_gqa(flags, R):
+    # 5 branches: the last query tile is ragged; 4 query heads share 2 kv heads; ragged caches
+    cfg = W.small(W.CONFIGS["cfg2"], S=2, B=5, R=R, Nc=300, Hq=4, Hkv=2)
+    attn = W.attention_inputs(cfg, DEV)
+    lens = torch.tensor([300, 173], dtype=torch.int32, device=DEV)
+    _check_attention(cfg, attn, flags, cache_lens=lens)
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_custom_visibility(flags):
+    # asymmetric visibility as in the inter-block variant (Section 3.4): drafts read the root
+    cfg = W.small(W.CONFIGS["cfg2"], S=2, B=7, R=32, Nc=128, Hq=2, Hkv=2)
+    vis = np.zeros((cfg.S, cfg.B, 1), dtype=np.int64)
+    vis[0, 1:, 0] = 1            # every draft of sequence 0 also reads branch 0
+    vis[1, 0, 0] = 0b1111111     # the root of sequence 1 reads everything
+    vis[1, 5, 0] = 0b0000110
+    _check_attention(cfg, W.attention_inputs(cfg, DEV), flags, vis=torch.from_numpy(vis).to(DEV))
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_no_cache_and_tiny_cache(flags):
+    for nc in (0, 16):
+        cfg = W.small(W.CONFIGS["cfg2"], B=4, Nc=nc, Hq=2, Hkv=2)
+        _check_attention(cfg, W.attention_inputs(cfg, DEV), flags)
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_poisoned_branches_do_not_leak(flags):
+    cfg = W.small(W.CONFIGS["cfg2"], B=8, Nc=256, Hq=2, Hkv=2)
+    clean = W.attention_inputs(cfg, DEV)
+    keep = 5
+    rows = slice(keep * cfg.R, (keep + 1) * cfg.R)
+    base, _ = _run_attention(cfg, clean, flags)
+    dirty, _ = _run_attention(cfg, W.poison_other_branches(cfg, clean, keep), flags)
+    # the kept branch cannot see the poisoned ones: bit-identical output
+    assert torch.equal(base.out[:, rows], dirty.out[:, rows])
+    assert dirty.out[:, rows].float().abs().max() < 10.0
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_sharp_scores(flags):
+    # queries scaled x4: near one-hot softmax rows, where a leaked or dropped key would show
+    cfg = W.small(W.CONFIGS["cfg2"], B=8, Nc=512, Hq=2, Hkv=2)
+    _check_attention(cfg, W.attention_inputs(cfg, DEV, q_gain=4.0), flags)
+
+
+@pytest.mark.parametrize("flags", PATHS)
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_attention_full_config(flags, name):
+    cfg = W.CONFIGS[name]
+    worst = _check_attention(cfg, W.attention_inputs(cfg, DEV), flags, heads=[0, 13, 31] if name == "cfg3" else None)
+    assert worst < 1e-2
+
+
+@pytest.mark.parametrize("name,seqs,heads", [("cfg4", [0, 15], [0, 31]), ("cfg5", [3], [0, 3])])
+def test_attention_full_size_sampled(name, seqs, heads):
+    # full-size launch as the benchmark times it; the oracle checks sampled (sequence, kv head) pairs
+    cfg = W.CONFIGS[name]
+    _check_attention(cfg, W.attention_inputs(cfg, DEV), 0, seqs=seqs, heads=heads)
+
+
+def test_attention_is_deterministic():
+    cfg = W.small(W.CONFIGS["cfg3"], Hq=4, Hkv=4)
+    attn = W.attention_inputs(cfg, DEV)
+    a, _ = _run_attention(cfg, attn, 0)
+    b, _ = _run_attention(cfg, attn, 0)
+    assert torch.equal(a.out, b.out) and torch.equal(a.attn_lse, b.attn_lse)
+
+
+# ----------------------------------------------------------------- confidence / top-k
+def _check_topk(logits, k, rows=None):
+    n, V = logits.shape
+    conf = torch.empty(n, dtype=torch.float32, device=DEV)
+    idx = torch.empty((n, k), dtype=torch.int32, device=DEV)
+    prob = torch.empty((n, k), dtype=torch.float32, device=DEV)
+    lse = torch.empty(n, dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, B.tsd_confidence_topk_workspace_bytes(n, V, k)), dtype=torch.uint8, device=DEV)
+    B.tsd_confidence_topk(logits, k, conf, idx, prob, lse, ws)
+    torch.cuda.synchronize()
+    sel = slice(None) if rows is None else torch.as_tensor(rows, device=DEV)
+    host = _np(logits[sel])
+    r_conf, r_idx, r_prob, r_lse = oracle.confidence_topk(host, k)
+    assert np.array_equal(idx[sel].cpu().numpy(), r_idx)
+    assert np.abs(conf[sel].cpu().numpy() - r_conf).max() <= 1e-5
+    assert np.abs(prob[sel].cpu().numpy() - r_prob).max() <= 1e-5
+    finite = np.isfinite(r_lse)
+    assert np.abs(lse[sel].cpu().numpy()[finite] - r_lse[finite]).max() <= 1e-4
+    return conf, idx, prob
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3"])
+def test_topk_full_config(name):
+    cfg = W.CONFIGS[name]
+    vi = W.verify_inputs(cfg, DEV)
+    _check_topk(vi["logits"], cfg.k)
+
+
+@pytest.mark.parametrize("name", ["cfg4", "cfg5"])
+def test_topk_full_size_sampled(name):
+    cfg = W.CONFIGS[name]
+    vi = W.verify_inputs(cfg, DEV)
+    rows = np.random.default_rng(1).choice(cfg.rows, 96, replace=False)
+    rows.sort()
+    _check_topk(vi["logits"], cfg.k, rows)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 5, 8])
+def test_topk_ragged_vocab_and_heavy_ties(dtype, k):
+    g = torch.Generator(device=DEV).manual_seed(k)
+    for n, V in ((7, 1000), (3, 40), (300, 2056), (5000, 520)):
+        # rounding to halves makes most of the top entries tie: index order decides
+        pitch = (V + 7) // 8 * 8 + 8          # rows padded: row pitch != vocabulary
+        buf = (torch.randn((n, pitch), generator=g, device=DEV) * 2).mul(2).round().div(2).to(dtype)
+        _check_topk(buf[:, :V], min(k, V))
+
+
+def test_topk_minus_inf_and_split_rows():
+    V = 126464
+    g = torch.Generator(device=DEV).manual_seed(5)
+    x = (torch.randn((6, V), generator=g, device=DEV) * 3).bfloat16()
+    x[0, :] = float("-inf")
+    x[0, 77] = 1.0                       # one finite entry: the rest tie at -inf, lowest indices first
+    x[1, 5:] = float("-inf")
+    x[2, V - 1] = 40.0                    # maximum in the last position of the last segment
+    x[3, 0] = 40.0
+    conf, idx, prob = _check_topk(x, 4)
+    assert idx[0].tolist() == [77, 0, 1, 2] and prob[0, 1] == 0
+
+
+def test_topk_is_deterministic():
+    cfg = W.CONFIGS["cfg2"]
+    vi = W.verify_inputs(cfg, DEV)
+    outs = []
+    for _ in range(3):
+        s = VerifyStep.for_config(cfg, DEV)
+        s.confidence_topk(vi["logits"])
+        torch.cuda.synchronize()
+        outs.append((s.conf.clone(), s.topk_idx.clone(), s.topk_prob.clone(), s.lse.clone()))
+    for o in outs[1:]:
+        assert all(torch.equal(a, b) for a, b in zip(outs[0], o))
+
+
+# ------------------------------------------------------------------------ acceptance
+def _gpu_accept(parent, state, mask_id, conf, top1, tau, rule, search, stride=1):
+    S, Bn, R = state.shape
+    t = lambda a, dt: torch.as_tensor(np.ascontiguousarray(a), dtype=dt, device=DEV)
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=DEV)
+    out = dict(edge_valid=e((S, Bn), torch.uint8), prefix_len=e((S, Bn), torch.int32),
+               accepted_node=e(S, torch.int32), accepted_len=e(S, torch.int32),
+               n_new_tokens=e(S, torch.int32), unmask_flag=e((S, R), torch.uint8),
+               unmask_tok=e((S, R), torch.int32))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.tsd_accept_trajectories(t(parent, torch.int32), t(state, torch.int32), mask_id, t(conf, torch.float32),
+                              t(top1, torch.int32), stride, tau, rule, search, status=status, **out)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}, status
+
+
+CASES = load_accept_cases()
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c["id"] for c in CASES])
+def test_accept_hand_worked_trees(case):
+    got, _ = _gpu_accept(case["parent"], case["state"], case["mask_id"], case["conf"], case["top1"],
+                         case["tau"], case["rule"], case["search"])
+    e = case["expect"]
+    for key in ("edge_valid", "prefix_len", "unmask_flag", "unmask_tok"):
+        assert got[key][0].tolist() == e[key], key
+    for key in ("accepted_node", "accepted_len", "n_new_tokens"):
+        assert int(got[key][0]) == e[key], key
+
+
+@pytest.mark.parametrize("R", [4, 32, 64, 100])
+def test_accept_random_trees_match_oracle(R):
+    rng = np.random.default_rng(R)
+    S, Bn, V = 33, 40, 50
+    M = V
+    parent = np.stack([[-1] + [int(rng.integers(0, b)) for b in range(1, Bn)] for _ in range(S)]).astype(np.int32)
+    conf = rng.random((S, Bn, R)).astype(np.float32)
+    conf[rng.random((S, Bn, R)) < 0.2] = 0.8           # exact ties with tau and among rows
+    top1 = rng.integers(0, V, (S, Bn, R)).astype(np.int32)
+    state = np.full((S, Bn, R), M, np.int32)
+    for s in range(S):
+        fill = rng.random(R) < 0.3
+        state[s, 0, fill] = rng.integers(0, V, fill.sum())
+        for b in range(1, Bn):
+            p = parent[s, b]
+            c = state[s, p].copy()
+            flag, tok = oracle.decode_rule(state[s, p], M, conf[s, p], top1[s, p], 0.8)
+            mode = rng.integers(0, 5)
+            rows = np.flatnonzero(c == M)
+            if mode <= 1:
+                c[flag.astype(bool)] = tok[flag.astype(bool)]
+            elif mode == 2 and len(rows):
+                r = rows[rng.integers(len(rows))]
+                c[r] = top1[s, p, r]
+            elif mode == 3 and len(rows):
+                c[rows[0]] = rng.integers(0, V)
+            elif mode == 4:
+                filled = np.flatnonzero(c != M)
+                if len(filled):
+                    c[filled[0]] = M if rng.random() < 0.5 else (c[filled[0]] + 1) % V   # malformed
+            state[s, b] = c
+    for rule in (0, 1):
+        for search in (0, 1):
+            ref = oracle.accept(parent, state, M, conf, top1, 0.8, rule, search)
+            got, status = _gpu_accept(parent, state, M, conf, top1, 0.8, rule, search)
+            for key, val in ref.items():
+                assert np.array_equal(got[key], val), (key, rule, search)
+            assert B.tsd_check_status(status) == B.TSD_OK
+
+
+def test_accept_reports_bad_parent_without_faulting():
+    parent = np.array([[-1, 0, 7, 1]], np.int32)       # node 2 points past itself
+    state = np.full((1, 4, 32), 9, np.int32)
+    conf = np.zeros((1, 4, 32), np.float32)
+    top1 = np.zeros((1, 4, 32), np.int32)
+    got, status = _gpu_accept(parent, state, 9, conf, top1, 0.9, 0, 0)
+    assert B.tsd_check_status(status) == B.TSD_ERR_DEVICE_DATA
+    assert got["edge_valid"][0, 2] == 0
+
+
+# ---------------------------------------------------------------- the whole hot path
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3"])
+def test_whole_step_matches_oracle(name):
+    cfg = W.CONFIGS[name]
+    attn = W.attention_inputs(cfg, DEV)
+    vi = W.verify_inputs(cfg, DEV)
+    step = VerifyStep.for_config(cfg, DEV)
+    res = step.run(attn, vi["logits"], vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
+    torch.cuda.synchronize()
+    step.check_status()
+    S, Bn, R = cfg.S, cfg.B, cfg.R
+    conf, idx, prob, _ = oracle.confidence_topk(_np(vi["logits"]), cfg.k)
+    assert np.array_equal(step.topk_idx.cpu().numpy(), idx)
+    g_conf = step.conf.cpu().numpy()
+    assert np.abs(g_conf - conf).max() <= 1e-5
+    # (a) same fp32 confidences on both sides: every decision bit-exact
+    same = oracle.accept(_np(vi["parent"]), _np(vi["state"]), vi["mask_id"], g_conf.reshape(S, Bn, R),
+                         idx[:, 0].reshape(S, Bn, R), cfg.tau)
+    # (b) the oracle's own chain (fp64 softmax rounded to fp32): the generator keeps confidences
+    # clear of tau and of each other, so the decisions agree as well
+    own = oracle.accept(_np(vi["parent"]), _np(vi["state"]), vi["mask_id"],
+                        conf.astype(np.float32).reshape(S, Bn, R), idx[:, 0].reshape(S, Bn, R), cfg.tau)
+    for key in same:
+        assert np.array_equal(res[key].cpu().numpy(), same[key]), key
+        assert np.array_equal(res[key].cpu().numpy(), own[key]), key
+    # the plan the generator planted is what the decoder found
+    assert int(res["edge_valid"].sum()) >= S
