@@ -286,18 +286,32 @@ def main():
     for st, _, _ in sets:
         st.check_status()
 
-    # ---------------- timed region B: each stage alone, back-to-back launches on rotating inputs
-    def time_stage(fn, reps):
-        for i in range(3):
-            fn(i)
+    # ---------------- timed region B: each stage alone, back-to-back launches on rotating inputs,
+    # replayed from a CUDA graph so that the host's launch cost does not set the pace
+    def time_stage(fn, min_seconds=0.25):
+        g = torch.cuda.CUDAGraph()
+        per_graph = max(n_copies, 4)
+        fn(0)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            for i in range(per_graph):
+                fn(i)
+        for _ in range(3):
+            g.replay()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
-        for i in range(reps):
-            fn(i)
+        g.replay()
         b.record(stream)
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps * 1e-3
+        once = max(a.elapsed_time(b) * 1e-3, 1e-6)
+        reps = int(min(max(min_seconds / once, 3), 20000))
+        a.record(stream)
+        for _ in range(reps):
+            g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e-3 / (reps * per_graph)
 
     def f_attn(i):
         step, attn, vi = sets[i % n_copies]
@@ -312,8 +326,7 @@ def main():
         step, attn, vi = sets[i % n_copies]
         step.accept(vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
 
-    reps = max(args.steps, 20)
-    t_attn, t_topk, t_acc = time_stage(f_attn, reps), time_stage(f_topk, reps), time_stage(f_acc, reps)
+    t_attn, t_topk, t_acc = time_stage(f_attn), time_stage(f_topk), time_stage(f_acc, 0.05)
     clocks = sampler.stop()
 
     # ---------------- end to end: pinned host inputs -> device -> step -> host results

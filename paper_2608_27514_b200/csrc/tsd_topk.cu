@@ -1,14 +1,21 @@
 // Stage 2: confidence and top-k candidates in one streaming pass over the logits
 // (paper Eq. 2: c = max softmax(logits); Section 3.2: top-k candidates per position).
 //
-// HBM-bound: every logit is read exactly once with 128-bit coalesced loads.  Each thread keeps a
-// running (max, sum of exp) pair and a sorted k-entry candidate list in registers; the hot loop
-// spends one compare against the list's last entry per element, so the insert path is rare.
-// Lists are merged by warp shuffles (k rounds of an arg-best reduction), then across the warps of
-// the block through shared memory.  With few rows a row is split into segments handled by
-// different blocks; the last block to finish a row (a ticket counter in the workspace, no
-// spinning) merges the segment partials in segment order, so the result does not depend on
-// arrival order.
+// HBM-bound, so the streaming loop is branch-free.  A block handles one row (or one segment of a
+// row when there are few rows) in three phases:
+//   1. stream: 128-bit coalesced loads, four chunks per thread in flight.  Per batch the thread
+//      takes the packed maximum of its 32 values, rebases its running sum to the new maximum with
+//      one multiply, adds 2^(x*log2e - e) for every value (one FFMA + one ex2 each), and stores the
+//      batch maximum in shared memory.
+//   2. bound: the k-th largest of the 256 per-thread maxima (warp shuffles, then across warps).
+//      At least k values of the row are >= it, so it is a valid lower bound of the k-th best.
+//   3. collect: each thread re-reads only those of its batches whose maximum reaches the bound
+//      (a handful per row, served by L2) and inserts the values >= bound into a sorted k-entry
+//      list in registers; lists are merged by warp shuffles (k rounds of an arg-best reduction),
+//      then across the warps of the block through shared memory.
+// With few rows a row is split into segments handled by different blocks; the last block to finish
+// a row (a ticket counter in the workspace, no spinning) merges the segment partials in segment
+// order, so the result does not depend on arrival order.
 //
 // Ordering is (logit descending, index ascending) on the raw input values (bf16 and fp32 both
 // widen to fp32 exactly), so indices are uniquely defined.
@@ -21,7 +28,9 @@ namespace tsd {
 
 constexpr int kTopkThreads = 256;
 constexpr int kTopkWarps = kTopkThreads / 32;
-constexpr int kTopkUnroll = 4;
+constexpr int kTopkUnroll = 4;                          // chunks per thread per batch
+constexpr int kTopkBatch = kTopkThreads * kTopkUnroll;  // chunks per block per batch
+constexpr int kTopkMaxIter = 32;                        // batches per segment (batch maxima kept in smem)
 constexpr int kMaxSegments = 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -42,22 +51,33 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return r;
 }
 
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// Sorted candidate list (key order) plus the row statistics that travel with it through merges:
+// the sum is kept as s * 2^e with e = fl(M * log2e) for the maximum M, so that one FFMA feeds
+// the exponential; the rounding of e is undone exactly in finalize().
 template <int K>
 struct Acc {
-  float v[K];  // candidate logits, sorted by key order
-  int i[K];    // their vocabulary indices
-  float m;     // v[0], or 0 while nothing finite has been seen (keeps x - m free of inf - inf)
-  float s;     // sum of exp(x - m) over the elements seen
+  float v[K];
+  int i[K];
+  float e;  // exponent base; meaningful only when `seen`
+  float s;
+  bool seen;  // a finite value contributed
 
   __device__ __forceinline__ void init() {
 #pragma unroll
     for (int j = 0; j < K; ++j) { v[j] = -CUDART_INF_F; i[j] = INT_MAX; }
-    m = 0.f;
+    e = 0.f;
     s = 0.f;
+    seen = false;
   }
-
-  // (x, xi) is known to come before the last entry: insert it, dropping the last.
-  __device__ __forceinline__ void insert(float x, int xi) {
+  // insert (x, xi) if it comes before the last entry
+  __device__ __forceinline__ void offer(float x, int xi) {
+    if (!key_before(x, xi, v[K - 1], i[K - 1])) return;
     bool placed = false;
 #pragma unroll
     for (int j = K - 1; j >= 1; --j) {
@@ -68,21 +88,6 @@ struct Acc {
     }
     if (!placed) { v[0] = x; i[0] = xi; }
   }
-
-  __device__ __forceinline__ void push(float x, int xi) {
-    if (x >= v[K - 1]) {  // rare once the list holds k large entries
-      if (key_before(x, xi, v[K - 1], i[K - 1])) {
-        if (x > v[0]) {  // new running maximum: rebase the sum
-          s *= ex2_approx((m - x) * kLog2e);
-          if (v[0] == -CUDART_INF_F) s = 0.f;
-          m = x;
-        }
-        insert(x, xi);
-      }
-    }
-    s += ex2_approx((x - m) * kLog2e);
-  }
-
   __device__ __forceinline__ void pop_front() {
 #pragma unroll
     for (int j = 0; j < K - 1; ++j) { v[j] = v[j + 1]; i[j] = i[j + 1]; }
@@ -95,10 +100,10 @@ struct Acc {
 template <int K>
 __device__ __forceinline__ void warp_merge(Acc<K>& a) {
   const unsigned full = 0xffffffffu;
-  float M = a.v[0];
+  float E = a.seen ? a.e : -CUDART_INF_F;
 #pragma unroll
-  for (int off = 16; off; off >>= 1) M = fmaxf(M, __shfl_xor_sync(full, M, off));
-  float s = (a.v[0] == -CUDART_INF_F) ? 0.f : a.s * ex2_approx((a.v[0] - M) * kLog2e);
+  for (int off = 16; off; off >>= 1) E = fmaxf(E, __shfl_xor_sync(full, E, off));
+  float s = a.seen ? a.s * ex2_approx(a.e - E) : 0.f;
 #pragma unroll
   for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(full, s, off);
   float ov[K];
@@ -120,12 +125,28 @@ __device__ __forceinline__ void warp_merge(Acc<K>& a) {
 #pragma unroll
   for (int r = 0; r < K; ++r) { a.v[r] = ov[r]; a.i[r] = oi[r]; }
   a.s = s;
-  a.m = (M == -CUDART_INF_F) ? 0.f : M;
+  a.seen = E != -CUDART_INF_F;
+  a.e = a.seen ? E : 0.f;
+}
+
+// k-th largest of the values held one per lane (K rounds; equal values leave together, which can
+// only lower the result, so it stays a valid lower bound).  Every lane gets the result.
+template <int K>
+__device__ __forceinline__ void warp_top_values(float x, float (&top)[K]) {
+  const unsigned full = 0xffffffffu;
+#pragma unroll
+  for (int r = 0; r < K; ++r) {
+    float b = x;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) b = fmaxf(b, __shfl_xor_sync(full, b, off));
+    top[r] = b;
+    if (x == b) x = -CUDART_INF_F;
+  }
 }
 
 template <int K>
 struct Partial {  // one segment's result, as stored in the workspace
-  float m, s;
+  float e, s;     // e = -inf when nothing finite was seen
   float v[K];
   int i[K];
 };
@@ -133,7 +154,10 @@ struct Partial {  // one segment's result, as stored in the workspace
 template <int K>
 __device__ __forceinline__ void finalize(const Acc<K>& a, int k, int64_t row, float* conf,
                                          int32_t* topk_idx, float* topk_prob, float* lse) {
-  const float M = a.v[0], Z = a.s;
+  // a.s = sum 2^(x*log2e - e) with e = fl(M*log2e): the FMA residual d = M*log2e - e is exact
+  const float M = a.v[0];
+  const float d = fmaf(M, kLog2e, -a.e);
+  const float Z = a.s * exp2f(-d);  // sum exp(x - M)
   const float inv = 1.f / Z;
 #pragma unroll
   for (int j = 0; j < K; ++j) {
@@ -152,27 +176,51 @@ struct Unpack;
 template <>
 struct Unpack<float> {
   static constexpr int kElems = 4;
-  template <int K>
-  static __device__ __forceinline__ void push(Acc<K>& a, const uint4& w, int base) {
-    a.push(__uint_as_float(w.x), base);
-    a.push(__uint_as_float(w.y), base + 1);
-    a.push(__uint_as_float(w.z), base + 2);
-    a.push(__uint_as_float(w.w), base + 3);
+  static constexpr uint32_t kNegInfWord = 0xff800000u;
+  static __device__ __forceinline__ float chunk_max(const uint4& w) {
+    return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)),
+                 fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
+  }
+  static __device__ __forceinline__ float batch_max(const uint4 (&b)[kTopkUnroll]) {
+    return fmaxf(fmaxf(chunk_max(b[0]), chunk_max(b[1])), fmaxf(chunk_max(b[2]), chunk_max(b[3])));
+  }
+  static __device__ __forceinline__ float elem(const uint4& w, int j) {
+    return __uint_as_float(j == 0 ? w.x : (j == 1 ? w.y : (j == 2 ? w.z : w.w)));
+  }
+  static __device__ __forceinline__ float sum_exp(const uint4& w, float ne, float s) {
+    s += ex2_approx(fmaf(__uint_as_float(w.x), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.y), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.z), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.w), kLog2e, ne));
+    return s;
   }
 };
 template <>
 struct Unpack<__nv_bfloat16> {
   static constexpr int kElems = 8;
-  template <int K>
-  static __device__ __forceinline__ void push(Acc<K>& a, const uint4& w, int base) {
-    a.push(__uint_as_float(w.x << 16), base);
-    a.push(__uint_as_float(w.x & 0xffff0000u), base + 1);
-    a.push(__uint_as_float(w.y << 16), base + 2);
-    a.push(__uint_as_float(w.y & 0xffff0000u), base + 3);
-    a.push(__uint_as_float(w.z << 16), base + 4);
-    a.push(__uint_as_float(w.z & 0xffff0000u), base + 5);
-    a.push(__uint_as_float(w.w << 16), base + 6);
-    a.push(__uint_as_float(w.w & 0xffff0000u), base + 7);
+  static constexpr uint32_t kNegInfWord = 0xff80ff80u;
+  static __device__ __forceinline__ float batch_max(const uint4 (&b)[kTopkUnroll]) {
+    uint32_t m = bmax2(bmax2(bmax2(b[0].x, b[0].y), bmax2(b[0].z, b[0].w)),
+                       bmax2(bmax2(b[1].x, b[1].y), bmax2(b[1].z, b[1].w)));
+    m = bmax2(m, bmax2(bmax2(bmax2(b[2].x, b[2].y), bmax2(b[2].z, b[2].w)),
+                       bmax2(bmax2(b[3].x, b[3].y), bmax2(b[3].z, b[3].w))));
+    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+  }
+  static __device__ __forceinline__ float elem(const uint4& w, int j) {
+    const uint32_t word = j < 2 ? w.x : (j < 4 ? w.y : (j < 6 ? w.z : w.w));
+    return __uint_as_float((j & 1) ? (word & 0xffff0000u) : (word << 16));
+  }
+  static __device__ __forceinline__ float sum_exp(const uint4& w, float ne, float s) {
+    // two partial sums per chunk keep the dependent add chain short
+    float s1 = ex2_approx(fmaf(__uint_as_float(w.x & 0xffff0000u), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.x << 16), kLog2e, ne));
+    s1 += ex2_approx(fmaf(__uint_as_float(w.y & 0xffff0000u), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.y << 16), kLog2e, ne));
+    s1 += ex2_approx(fmaf(__uint_as_float(w.z & 0xffff0000u), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.z << 16), kLog2e, ne));
+    s1 += ex2_approx(fmaf(__uint_as_float(w.w & 0xffff0000u), kLog2e, ne));
+    s += ex2_approx(fmaf(__uint_as_float(w.w << 16), kLog2e, ne));
+    return s + s1;
   }
 };
 
@@ -184,6 +232,9 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
                        float* __restrict__ topk_prob, float* __restrict__ lse,
                        Partial<K>* __restrict__ partials, unsigned* __restrict__ tickets) {
   constexpr int E = Unpack<T>::kElems;
+  __shared__ float s_bmax[kTopkMaxIter][kTopkThreads];  // per-thread batch maxima
+  __shared__ float s_top[kTopkWarps][K];
+  __shared__ Partial<K> s_part[kTopkWarps];
   const int64_t row = blockIdx.x / n_seg;
   const int seg = blockIdx.x % n_seg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -192,41 +243,113 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   const int chunks_total = vocab / E;
   const int c0 = seg * chunks_per_seg;
   const int c1 = min(c0 + chunks_per_seg, chunks_total);
+  const int n_iter = (c1 - c0 + kTopkBatch - 1) / kTopkBatch;  // <= kTopkMaxIter (host-enforced)
+  const bool has_tail = seg == n_seg - 1 && tid == 0 && chunks_total * E < vocab;
 
-  Acc<K> a;
-  a.init();
-  for (int base = c0 + tid; base < c1; base += kTopkThreads * kTopkUnroll) {
+  // ---- phase 1: stream
+  float m = -CUDART_INF_F, e = 0.f, s = 0.f;
+  for (int it = 0; it < n_iter; ++it) {
+    const int base = c0 + it * kTopkBatch + tid;
     uint4 buf[kTopkUnroll];
 #pragma unroll
     for (int u = 0; u < kTopkUnroll; ++u) {
       const int c = base + u * kTopkThreads;
       if (c < c1) buf[u] = ld_stream(rowv + c);
+      else  // past the segment: -inf adds nothing and is never a candidate
+        buf[u] = make_uint4(Unpack<T>::kNegInfWord, Unpack<T>::kNegInfWord, Unpack<T>::kNegInfWord,
+                            Unpack<T>::kNegInfWord);
     }
+    const float bm = Unpack<T>::batch_max(buf);
+    s_bmax[it][tid] = bm;
+    const float m_new = fmaxf(m, bm);
+    const float e_new = (m_new == -CUDART_INF_F) ? 0.f : m_new * kLog2e;
+    s *= (m == -CUDART_INF_F) ? 0.f : ex2_approx(e - e_new);  // rebase: 1 when the maximum stays
+    m = m_new;
+    e = e_new;
 #pragma unroll
+    for (int u = 0; u < kTopkUnroll; ++u) s = Unpack<T>::sum_exp(buf[u], -e, s);
+  }
+  float tail_max = -CUDART_INF_F;
+  if (has_tail) {  // ragged tail of a vocabulary that is not a multiple of the chunk size
+    for (int x = chunks_total * E; x < vocab; ++x) tail_max = fmaxf(tail_max, to_float(rowp[x]));
+    const float m_new = fmaxf(m, tail_max);
+    const float e_new = (m_new == -CUDART_INF_F) ? 0.f : m_new * kLog2e;
+    s *= (m == -CUDART_INF_F) ? 0.f : ex2_approx(e - e_new);
+    m = m_new;
+    e = e_new;
+    for (int x = chunks_total * E; x < vocab; ++x) s += ex2_approx(fmaf(to_float(rowp[x]), kLog2e, -e));
+  }
+
+  // ---- phase 2: bound = k-th largest per-thread maximum of the block
+  float top[K];
+  warp_top_values<K>(m, top);
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < K; ++j) s_top[warp][j] = top[j];
+  }
+  __syncthreads();
+  {
+    // every warp redoes the small cross-warp step: lanes hold the 8 x K warp values
+    float x = -CUDART_INF_F, bound = -CUDART_INF_F;
+    // K rounds over up to 32 candidate values per round-robin slice (8*K <= 64)
+    float c0v = lane < kTopkWarps * K ? s_top[lane / K][lane % K] : -CUDART_INF_F;
+    float c1v = lane + 32 < kTopkWarps * K ? s_top[(lane + 32) / K][(lane + 32) % K] : -CUDART_INF_F;
+#pragma unroll
+    for (int r = 0; r < K; ++r) {
+      x = fmaxf(c0v, c1v);
+#pragma unroll
+      for (int off = 16; off; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, off));
+      bound = x;
+      if (c0v == x) c0v = -CUDART_INF_F;
+      if (c1v == x) c1v = -CUDART_INF_F;
+    }
+    top[0] = bound;
+  }
+  const float bound = top[0];
+
+  // ---- phase 3: collect the values >= bound from the few batches that hold one
+  Acc<K> a;
+  a.init();
+  a.seen = m != -CUDART_INF_F;
+  a.e = e;
+  a.s = s;
+  for (int it = 0; it < n_iter; ++it) {
+    if (!(s_bmax[it][tid] >= bound)) continue;
+#pragma unroll 1
     for (int u = 0; u < kTopkUnroll; ++u) {
-      const int c = base + u * kTopkThreads;
-      if (c < c1) Unpack<T>::push(a, buf[u], c * E);
+      const int c = c0 + it * kTopkBatch + tid + u * kTopkThreads;
+      if (c >= c1) break;
+      const uint4 w = rowv[c];
+#pragma unroll 1
+      for (int j = 0; j < E; ++j) {
+        const float x = Unpack<T>::elem(w, j);
+        if (x >= bound) a.offer(x, c * E + j);
+      }
     }
   }
-  if (seg == n_seg - 1 && tid == 0) {  // ragged tail of a vocabulary that is not a multiple of E
-    for (int x = chunks_total * E; x < vocab; ++x) a.push(to_float(rowp[x]), x);
+  if (has_tail && tail_max >= bound) {
+    for (int x = chunks_total * E; x < vocab; ++x) {
+      const float v = to_float(rowp[x]);
+      if (v >= bound) a.offer(v, x);
+    }
   }
 
   warp_merge(a);
-  __shared__ Partial<K> sm[kTopkWarps];
   if (lane == 0) {
-    sm[warp].m = a.v[0];
-    sm[warp].s = a.s;
+    s_part[warp].e = a.seen ? a.e : -CUDART_INF_F;
+    s_part[warp].s = a.s;
 #pragma unroll
-    for (int j = 0; j < K; ++j) { sm[warp].v[j] = a.v[j]; sm[warp].i[j] = a.i[j]; }
+    for (int j = 0; j < K; ++j) { s_part[warp].v[j] = a.v[j]; s_part[warp].i[j] = a.i[j]; }
   }
   __syncthreads();
   if (warp != 0) return;
   a.init();
   if (lane < kTopkWarps) {
-    a.s = sm[lane].s;
+    a.seen = s_part[lane].e != -CUDART_INF_F;
+    a.e = a.seen ? s_part[lane].e : 0.f;
+    a.s = s_part[lane].s;
 #pragma unroll
-    for (int j = 0; j < K; ++j) { a.v[j] = sm[lane].v[j]; a.i[j] = sm[lane].i[j]; }
+    for (int j = 0; j < K; ++j) { a.v[j] = s_part[lane].v[j]; a.i[j] = s_part[lane].i[j]; }
   }
   warp_merge(a);
   if (n_seg == 1) {
@@ -237,7 +360,7 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   unsigned ticket = 0;
   if (lane == 0) {
     Partial<K>* p = partials + row * n_seg + seg;
-    p->m = a.v[0];
+    p->e = a.seen ? a.e : -CUDART_INF_F;
     p->s = a.s;
 #pragma unroll
     for (int j = 0; j < K; ++j) { p->v[j] = a.v[j]; p->i[j] = a.i[j]; }
@@ -250,6 +373,9 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   a.init();
   if (lane < n_seg) {
     const Partial<K>* p = partials + row * n_seg + lane;
+    const float pe = __ldcg(&p->e);
+    a.seen = pe != -CUDART_INF_F;
+    a.e = a.seen ? pe : 0.f;
     a.s = __ldcg(&p->s);
 #pragma unroll
     for (int j = 0; j < K; ++j) { a.v[j] = __ldcg(&p->v[j]); a.i[j] = __ldcg(&p->i[j]); }
@@ -273,6 +399,9 @@ static TopkPlan topk_plan(int64_t n_rows, int vocab, int k, int elems_per_chunk)
   int64_t n_seg = n_rows >= target_units ? 1 : (target_units + n_rows - 1) / n_rows;
   n_seg = std::min<int64_t>(n_seg, kMaxSegments);
   n_seg = std::min<int64_t>(n_seg, std::max(1, chunks / 1024));
+  // a segment may span at most kTopkMaxIter batches (its batch maxima live in shared memory)
+  const int64_t seg_cap = (int64_t)kTopkBatch * kTopkMaxIter;
+  n_seg = std::max<int64_t>(n_seg, (chunks + seg_cap - 1) / seg_cap);
   p.n_seg = (int)std::max<int64_t>(n_seg, 1);
   p.chunks_per_seg = (chunks + p.n_seg - 1) / p.n_seg;
   if (p.chunks_per_seg == 0) p.chunks_per_seg = 1;
@@ -320,6 +449,9 @@ extern "C" {
 static int topk_check(int64_t n_rows, int32_t vocab, int32_t k) {
   if (n_rows < 0 || vocab < 1 || k < 1 || k > 8 || k > vocab) return TSD_ERR_INVALID_ARG;
   if (n_rows * (int64_t)tsd::kMaxSegments > 0x7fffffffLL) return TSD_ERR_INVALID_ARG;
+  // rows longer than kMaxSegments segments of kTopkMaxIter batches (4 Mi fp32 / 8 Mi bf16 logits)
+  if ((int64_t)vocab / 4 > (int64_t)tsd::kTopkBatch * tsd::kTopkMaxIter * tsd::kMaxSegments)
+    return TSD_ERR_INVALID_ARG;
   return TSD_OK;
 }
 

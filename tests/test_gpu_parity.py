@@ -341,3 +341,19 @@ def test_whole_step_matches_oracle(name):
         assert np.array_equal(res[key].cpu().numpy(), own[key]), key
     # the plan the generator planted is what the decoder found
     assert int(res["edge_valid"].sum()) >= S
+
+
+def test_topk_subnormal_and_signed_zero_logits():
+    # thresholds that sit at +-0 or at subnormal bf16 values must still order exactly
+    V = 4096
+    x = torch.full((4, V), -1.0, dtype=torch.bfloat16, device=DEV)
+    tiny = torch.tensor([1e-40], dtype=torch.float32).bfloat16().item()   # a subnormal bf16
+    x[0, 100], x[0, 2000], x[0, 3000], x[0, 50] = 0.0, -0.0, tiny, 2 * tiny
+    x[1, :] = -0.0
+    x[1, 3000] = 0.0
+    x[2, :] = tiny
+    x[2, 7] = 2 * tiny
+    x[2, 4000] = 3 * tiny
+    x[3, :] = -tiny
+    x[3, 9], x[3, 10] = -0.0, 0.0
+    _check_topk(x, 4)
