@@ -8,9 +8,15 @@
 //
 // Warp roles: warps 0-3 = softmax (one query row per thread, TMEM lane = row), warp 4 = TMA
 // producer, warp 5 = tcgen05 MMA issuer (also owns the TMEM allocation).
-//   S = Q K^T : tcgen05.mma, A and B K-major from 128B-swizzled shared memory, fp32 in TMEM (x2 buffers)
-//   softmax  : tcgen05.ld S -> registers, running max / sum in the exp2 domain, P -> bf16 -> shared
-//   O += P V : tcgen05.mma, A = P (K-major), B = V (MN-major: head_dim contiguous), fp32 in TMEM
+//   S = Q K^T : tcgen05.mma, A and B K-major from 128B-swizzled shared memory, fp32 in TMEM
+//   softmax  : tcgen05.ld S -> registers, running max / sum in the exp2 domain, P -> bf16 -> TMEM
+//              (tcgen05.st over the first 32 columns of that S buffer: two bf16 per 32-bit column)
+//   O += P V : tcgen05.mma, A = P from TMEM, B = V (MN-major: head_dim contiguous), fp32 in TMEM
+// Key tiles are 64 keys wide.  S is double-buffered in TMEM (2 x 64 columns) so that Q K^T of tile
+// j+1 runs while the softmax of tile j is on the CUDA cores, and two blocks share an SM (each 256 of
+// the 512 TMEM columns and ~97 KB of shared memory) so that one block's P V fills the gaps of the
+// other.  MMAs issued by one thread execute in order, so an S/P buffer may be overwritten by a later
+// Q K^T as soon as the P V that reads it has been issued.
 // The running maximum used as exponent offset only moves when the row maximum grows by more than
 // 2^8, so rescaling O in TMEM is rare; the final division by the row sum makes the result exact.
 // Every mbarrier wait is bounded: on expiry the block raises TSD_STATUS_TIMEOUT, stops issuing
@@ -25,15 +31,21 @@ namespace tsd {
 constexpr int kTcThreads = 192;
 constexpr uint32_t kSub = 16384;          // bytes of one [128 rows x 64 elements] bf16 sub-tile
 constexpr uint32_t kTileBytes = 2 * kSub;  // a [128 x 128] bf16 tile
-constexpr uint32_t kOffQ = 0, kOffP = kTileBytes, kOffK = 2 * kTileBytes, kOffV = 4 * kTileBytes;
-constexpr uint32_t kOffBar = 6 * kTileBytes;
+constexpr int kKeys = 64;                       // keys per tile
+constexpr uint32_t kSubKV = 8192;              // bytes of one [64 keys x 64 elements] bf16 sub-tile
+constexpr uint32_t kKVBytes = 2 * kSubKV;      // a [64 x 128] bf16 K or V tile
+constexpr uint32_t kOffQ = 0, kOffK = kTileBytes, kOffV = kTileBytes + 2 * kKVBytes;  // 2 stages each
+constexpr uint32_t kOffBar = kTileBytes + 4 * kKVBytes;
+constexpr uint32_t kColS = 0, kColO = 128;     // S buffers at columns 0 and 64; P aliases 32 columns of each
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + slack to align the base to 1 KB
 constexpr uint32_t kSpinLimit = 1u << 21;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-enum Bar { Q_FULL = 0, K_FULL = 1, K_EMPTY = 3, V_FULL = 5, V_EMPTY = 7, S_FULL = 9, S_EMPTY = 11,
-           P_FULL = 13, PV_DONE = 14, N_BARS = 15 };
+// S_FULL[b] (Q K^T of a tile complete) also frees that tile's K stage; PV_DONE[b] (P V complete)
+// also frees its V stage: a tcgen05.commit costs ~100 clocks of the issuing thread, so each event
+// gets exactly one.
+enum Bar { Q_FULL = 0, K_FULL = 1, V_FULL = 3, S_FULL = 5, P_FULL = 7, PV_DONE = 9, N_BARS = 11 };
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -53,10 +65,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false when the block is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// The non-blocking test comes first: a phase that has already completed costs one shared-memory
+// round trip instead of a suspend / wake-up.
+// `sleep_ns` > 0 backs off between polls: used by the roles that run far ahead (the TMA producer),
+// whose spinning would otherwise take issue slots from the softmax warps on the same scheduler.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t sleep_ns = 0) {
+  if (mbar_test_wait(bar, parity)) return true;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (sleep_ns) __nanosleep(sleep_ns);
     if ((it & 255u) == 255u && *abort_flag) return false;
   }
   *abort_flag = 1u;
@@ -70,6 +95,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+// True in exactly one lane of a converged warp; the compiler recognises the pattern and keeps the
+// warp's address arithmetic on the uniform datapath, which the tcgen05 instructions read.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\n@p mov.u32 %0, 1;\n}" : "+r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -77,11 +110,30 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+// ACC is a compile-time constant so that the accumulate predicate costs nothing at issue time; the
+// issue rate of the elected thread is what keeps the tensor pipe fed (64 clocks per 128x128x16 MMA).
+template <bool ACC>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  if (ACC)
+    asm volatile("{\n.reg .pred p;\nsetp.eq.b32 p, 0, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+  else
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, 0, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+}
+
+template <bool ACC>
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+  if (ACC)
+    asm volatile("{\n.reg .pred p;\nsetp.eq.b32 p, 0, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc) : "memory");
+  else
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, 0, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc) : "memory");
 }
 
 #define TSD_R32(a, o) "=r"(a[o+0]), "=r"(a[o+1]), "=r"(a[o+2]), "=r"(a[o+3]), "=r"(a[o+4]), "=r"(a[o+5]), "=r"(a[o+6]), "=r"(a[o+7]), \
@@ -118,14 +170,64 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return r;
 }
 
+// Packed fp32 pairs (two lanes per instruction on this architecture) and the 3-input maximum.
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi) { return pack2(__float_as_uint(lo), __float_as_uint(hi)); }
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// 2^t for a pair, t in [-126, 16], on the FMA pipe: t = n + f with n = round(t), f in [-0.5, 0.5];
+// 2^f by a degree-3 polynomial (relative error 7.5e-5, well below the bf16 rounding of P), and n
+// added into the exponent field.  Takes load off the 16-per-clock special-function unit.
+__device__ __forceinline__ void exp2_poly2(uint64_t t2, float& p0, float& p1) {
+  float t0, t1;
+  unpack2(t2, t0, t1);
+  t2 = pack2f(fmaxf(t0, -126.f), fmaxf(t1, -126.f));
+  const uint64_t magic = pack2f(12582912.f, 12582912.f);          // 1.5 * 2^23: rounds to an integer
+  const uint64_t y = add2(t2, magic);
+  const uint64_t n = add2(y, pack2f(-12582912.f, -12582912.f));
+  const uint64_t f = fma2(n, pack2f(-1.f, -1.f), t2);
+  uint64_t r = fma2(f, pack2f(0.05517165f, 0.05517165f), pack2f(0.24261113f, 0.24261113f));
+  r = fma2(r, f, pack2f(0.69326097f, 0.69326097f));
+  r = fma2(r, f, pack2f(0.99992806f, 0.99992806f));
+  float y0, y1, r0, r1;
+  unpack2(y, y0, y1);
+  unpack2(r, r0, r1);
+  p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(y0) << 23));
+  p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(y1) << 23));
+}
+constexpr int kPolyOf8 = 2;  // of every 8 score pairs, this many take the polynomial exp2 (unmasked tiles)
+
 // Shared-memory matrix descriptor, 128-byte swizzle (descriptor version 1 = this architecture).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = N = 128; b_mn = 1 when B is MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(uint32_t b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n; b_mn = 1 when B is MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(uint32_t n, uint32_t b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 struct TcParams {
@@ -138,7 +240,7 @@ struct TcParams {
   float scale_log2e;  // sm_scale * log2(e), > 0
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                     const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kd,
                     const __grid_constant__ CUtensorMap map_vd, const TcParams p) {
@@ -163,9 +265,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   }
   const int clen = mask[kHdrWords + s];
   const int32_t* rec = mask + mask[H_RECS_OFF] + (size_t)(s * mask[H_NQT] + qt) * mask[H_REC_WORDS];
-  const int n_ct = (clen + kTile - 1) / kTile;  // cached tiles
-  const int n_dt = rec[0];                      // visible draft tiles
-  const int T = n_ct + n_dt;
+  const int n_ct = (clen + kKeys - 1) / kKeys;  // cached tiles of 64 keys
+  const int n_dt = rec[0];                      // visible 128-row draft tiles = 2 key tiles each
+  const int T = n_ct + 2 * n_dt;
 
   if (tid == 0) {
     abort_flag[0] = 0;
@@ -173,19 +275,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     mbar_init(bar(Q_FULL), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(K_FULL + i), 1);
-      mbar_init(bar(K_EMPTY + i), 1);
       mbar_init(bar(V_FULL + i), 1);
-      mbar_init(bar(V_EMPTY + i), 1);
       mbar_init(bar(S_FULL + i), 1);
-      mbar_init(bar(S_EMPTY + i), 4);
+      mbar_init(bar(P_FULL + i), 4);
+      mbar_init(bar(PV_DONE + i), 1);
     }
-    mbar_init(bar(P_FULL), 4);
-    mbar_init(bar(PV_DONE), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  if (warp == 5) {  // TMEM: 2 x S (128 columns each) + O (128 columns) -> 512-column allocation
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(bars + 128u) : "memory");
+  if (warp == 5) {  // TMEM: 2 x S/P (64 columns each) + O (128 columns); two blocks share the SM's 512
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(bars + 128u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -197,12 +296,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ------------------------------------------------------------ TMA producer (one lane)
     if (lane == 0) {
       auto load_tile = [&](uint32_t dst, uint32_t full_bar, const CUtensorMap* mc, const CUtensorMap* md, int j) {
-        mbar_expect_tx(full_bar, kTileBytes);
+        mbar_expect_tx(full_bar, kKVBytes);
         const bool cached = j < n_ct;
         const CUtensorMap* m = cached ? mc : md;
-        const int row = cached ? j * kTile : rec[2 + 2 * (j - n_ct)] * kTile;
+        const int e = j - n_ct;  // draft key tile e = half (e & 1) of the listed 128-row tile e >> 1
+        const int row = cached ? j * kKeys : rec[2 + 2 * (e >> 1)] * kTile + (e & 1) * kKeys;
         tma_load_4d(dst, m, full_bar, 0, g, row, s);
-        tma_load_4d(dst + kSub, m, full_bar, 64, g, row, s);
+        tma_load_4d(dst + kSubKV, m, full_bar, 64, g, row, s);
       };
       mbar_expect_tx(bar(Q_FULL), kTileBytes);
       tma_load_4d(base + kOffQ, &map_q, bar(Q_FULL), 0, h, qt * kTile, s);
@@ -210,12 +310,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       bool ok = true;
       int k_issued = 0, v_issued = 0;
       auto load_k = [&](int j) {
-        if (j >= 2) ok = ok && mbar_wait(bar(K_EMPTY + (j & 1)), ((j >> 1) - 1) & 1, abort_flag);
-        if (ok) { load_tile(base + kOffK + (j & 1) * kTileBytes, bar(K_FULL + (j & 1)), &map_kc, &map_kd, j); k_issued = j + 1; }
+        if (j >= 2) ok = ok && mbar_wait(bar(S_FULL + (j & 1)), ((j >> 1) - 1) & 1, abort_flag, 100);
+        if (ok) { load_tile(base + kOffK + (j & 1) * kKVBytes, bar(K_FULL + (j & 1)), &map_kc, &map_kd, j); k_issued = j + 1; }
       };
       auto load_v = [&](int j) {
-        if (j >= 2) ok = ok && mbar_wait(bar(V_EMPTY + (j & 1)), ((j >> 1) - 1) & 1, abort_flag);
-        if (ok) { load_tile(base + kOffV + (j & 1) * kTileBytes, bar(V_FULL + (j & 1)), &map_vc, &map_vd, j); v_issued = j + 1; }
+        if (j >= 2) ok = ok && mbar_wait(bar(PV_DONE + (j & 1)), ((j >> 1) - 1) & 1, abort_flag, 100);
+        if (ok) { load_tile(base + kOffV + (j & 1) * kKVBytes, bar(V_FULL + (j & 1)), &map_vc, &map_vd, j); v_issued = j + 1; }
       };
       if (T > 0) load_k(0);
       for (int j = 0; j < T && ok; ++j) {
@@ -230,49 +330,84 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------ MMA issuer (one lane)
-    if (lane == 0) {
-      const uint32_t idesc_qk = instr_desc(0), idesc_pv = instr_desc(1);
+    // ------------------------------------------------------------ MMA issuer
+    // The whole warp walks the loop (uniform control flow, all lanes wait on the barriers); one
+    // elected lane issues the MMAs and commits.
+    {
+      constexpr uint32_t idesc_qk = instr_desc(kKeys, 0), idesc_pv = instr_desc(128, 1);
       bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
-      for (int j = 0; j <= T && ok; ++j) {
-        if (j < T) {  // S[j&1] = Q K_j^T
-          const int b = j & 1;
-          ok = ok && mbar_wait(bar(K_FULL + b), (j >> 1) & 1, abort_flag);
-          if (j >= 2) ok = ok && mbar_wait(bar(S_EMPTY + b), ((j >> 1) - 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t qa = base + kOffQ, ka = base + kOffK + b * kTileBytes;
+      // Every operand is built once, from values the compiler can see are warp-uniform (a lane-0
+      // broadcast), and kept in registers: descriptors differ only in their 14-bit address field.
+      const uint32_t ubase = __shfl_sync(0xffffffffu, base, 0);
+      const uint32_t utmem = __shfl_sync(0xffffffffu, tmem, 0);
+      uint64_t qd[8], kd[2][8], vd[2][kKeys / 16];
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t off = (kk >> 2) * kSub + (kk & 3) * 32;
-            tc_mma(tmem + b * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), idesc_qk, kk > 0);
+      for (int kk = 0; kk < 8; ++kk) {
+        qd[kk] = smem_desc(ubase + kOffQ + (kk >> 2) * kSub + (kk & 3) * 32, 16, 1024);
+#pragma unroll
+        for (int b = 0; b < 2; ++b)
+          kd[b][kk] = smem_desc(ubase + kOffK + b * kKVBytes + (kk >> 2) * kSubKV + (kk & 3) * 32, 16, 1024);
+      }
+#pragma unroll
+      for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int kk = 0; kk < kKeys / 16; ++kk)
+          vd[b][kk] = smem_desc(ubase + kOffV + b * kKVBytes + kk * 2048, kSubKV, 1024);
+      // S[j&1] = Q K_j^T (8 MMAs of K = 16 over head_dim).  The buffer was last read by P V of tile
+      // j-2, which was issued earlier, so in-order execution makes it safe to overwrite.
+      auto issue_qk = [&](int j) {
+        const int b = j & 1;
+        ok = ok && mbar_wait(bar(K_FULL + b), (j >> 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) return;
+        tc_fence_after();
+        if (elect_one()) {
+          if (b == 0) {
+            tc_mma<false>(utmem + kColS, qd[0], kd[0][0], idesc_qk);
+#pragma unroll
+            for (int kk = 1; kk < 8; ++kk) tc_mma<true>(utmem + kColS, qd[kk], kd[0][kk], idesc_qk);
+          } else {
+            tc_mma<false>(utmem + kColS + kKeys, qd[0], kd[1][0], idesc_qk);
+#pragma unroll
+            for (int kk = 1; kk < 8; ++kk) tc_mma<true>(utmem + kColS + kKeys, qd[kk], kd[1][kk], idesc_qk);
           }
           tc_commit(bar(S_FULL + b));
-          tc_commit(bar(K_EMPTY + b));
         }
-        if (j >= 1) {  // O += P_{j-1} V_{j-1}
-          const int jj = j - 1, b = jj & 1;
-          ok = ok && mbar_wait(bar(V_FULL + b), (jj >> 1) & 1, abort_flag);
-          ok = ok && mbar_wait(bar(P_FULL), jj & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t pa = base + kOffP, va = base + kOffV + b * kTileBytes;
+        __syncwarp();
+      };
+      if (ok && T > 0) issue_qk(0);
+      for (int j = 0; j < T && ok; ++j) {
+        if (j + 1 < T) issue_qk(j + 1);  // runs while the softmax of tile j is on the CUDA cores
+        // O += P_j V_j: P from TMEM (16 keys = 8 packed columns per MMA), V MN-major from shared memory
+        const int b = j & 1;
+        ok = ok && mbar_wait(bar(V_FULL + b), (j >> 1) & 1, abort_flag);
+        ok = ok && mbar_wait(bar(P_FULL + b), (j >> 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        if (elect_one()) {
+          if (j == 0) {
+            tc_mma_ts<false>(utmem + kColO, utmem + kColS, vd[0][0], idesc_pv);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t a_off = (kk >> 2) * kSub + (kk & 3) * 32;
-            tc_mma(tmem + 256, smem_desc(pa + a_off, 16, 1024), smem_desc(va + kk * 2048, kSub, 1024), idesc_pv,
-                   (jj > 0 || kk > 0));
+            for (int kk = 1; kk < kKeys / 16; ++kk) tc_mma_ts<true>(utmem + kColO, utmem + kColS + kk * 8, vd[0][kk], idesc_pv);
+          } else if (b == 0) {
+#pragma unroll
+            for (int kk = 0; kk < kKeys / 16; ++kk) tc_mma_ts<true>(utmem + kColO, utmem + kColS + kk * 8, vd[0][kk], idesc_pv);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < kKeys / 16; ++kk)
+              tc_mma_ts<true>(utmem + kColO, utmem + kColS + kKeys + kk * 8, vd[1][kk], idesc_pv);
           }
-          tc_commit(bar(PV_DONE));
-          tc_commit(bar(V_EMPTY + b));
+          tc_commit(bar(PV_DONE + b));
         }
+        __syncwarp();
       }
     }
   } else {
     // ------------------------------------------------------------ softmax, one query row per thread
     const int r = tid;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-    const int slots = kTile / p.R, qs = r / p.R;
+    const int qs = r / p.R;
     const float c = p.scale_log2e;
     float m_used = -CUDART_INF_F, l = 0.f;
     bool ok = true;
@@ -282,95 +417,106 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = __all_sync(0xffffffffu, ok);  // leave the loop as a whole warp
       if (!ok) break;
       tc_fence_after();
-      uint32_t sv[128];
-      TSD_TMEM_LD32(sv, 0, t_lane + b * 128);
-      TSD_TMEM_LD32(sv, 32, t_lane + b * 128 + 32);
-      TSD_TMEM_LD32(sv, 64, t_lane + b * 128 + 64);
-      TSD_TMEM_LD32(sv, 96, t_lane + b * 128 + 96);
+      const uint32_t t_s = t_lane + kColS + b * kKeys;
+      uint32_t sv[kKeys];
+      TSD_TMEM_LD32(sv, 0, t_s);
+      TSD_TMEM_LD32(sv, 32, t_s + 32);
       tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(S_EMPTY + b));  // S is in registers: the buffer may be overwritten
 
-      // visibility of this tile's 128 keys for this row
-      uint32_t cm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+      // visibility of this tile's 64 keys for this row
+      uint32_t cm[2] = {0xffffffffu, 0xffffffffu};
       bool masked = false;
       if (j < n_ct) {
-        const int valid = clen - j * kTile;  // keys past the sequence's cache length are invisible
-        if (valid < kTile) {
+        const int valid = clen - j * kKeys;  // keys past the sequence's cache length are invisible
+        if (valid < kKeys) {
           masked = true;
 #pragma unroll
-          for (int w = 0; w < 4; ++w) {
+          for (int w = 0; w < 2; ++w) {
             const int v = valid - 32 * w;
             cm[w] = v >= 32 ? 0xffffffffu : (v <= 0 ? 0u : ((1u << v) - 1u));
           }
         }
       } else {
-        const uint32_t nib = ((uint32_t)rec[3 + 2 * (j - n_ct)] >> (qs * 4)) & 15u;
+        const int e = j - n_ct;
+        const uint32_t nib = ((uint32_t)rec[3 + 2 * (e >> 1)] >> (qs * 4)) & 15u;  // visible key slots
         masked = true;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) cm[w] = ((nib >> ((w * 32) / p.R)) & 1u) ? 0xffffffffu : 0u;
-        (void)slots;
+        for (int w = 0; w < 2; ++w) cm[w] = ((nib >> (((e & 1) * kKeys + w * 32) / p.R)) & 1u) ? 0xffffffffu : 0u;
       }
       if (masked) {
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < kKeys; ++i)
           if (!((cm[i >> 5] >> (i & 31)) & 1u)) sv[i] = 0xff800000u;  // -inf: weight exactly 0
       }
       float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};  // independent chains
 #pragma unroll
-      for (int i = 0; i < 128; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sv[i]));
+      for (int i = 0; i < kKeys / 2; ++i)
+        mx4[i & 3] = max3(mx4[i & 3], __uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1]));
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m_used, mx * c);
       const bool grow = m_new > m_used + 8.f;  // also true for the first finite maximum
       const float alpha = grow ? ex2f(m_used - m_new) : 1.f;
       if (grow) m_used = m_new;
       const float off = (m_used == -CUDART_INF_F) ? 0.f : -m_used;
-      float rs4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pk[64];
+      const uint64_t c2 = pack2f(c, c), off2 = pack2f(off, off);
+      uint64_t rs4[4] = {0ull, 0ull, 0ull, 0ull};
+      uint32_t pk[kKeys / 2];
+      if (masked) {  // every exponential on the special-function unit: 2^(-inf) is exactly 0
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float p0 = ex2f(fmaf(__uint_as_float(sv[2 * i]), c, off));
-        const float p1 = ex2f(fmaf(__uint_as_float(sv[2 * i + 1]), c, off));
-        rs4[i & 3] += p0 + p1;
-        pk[i] = pack_bf16x2(p0, p1);
+        for (int i = 0; i < kKeys / 2; ++i) {
+          float t0, t1;
+          unpack2(fma2(pack2(sv[2 * i], sv[2 * i + 1]), c2, off2), t0, t1);
+          const float p0 = ex2f(t0), p1 = ex2f(t1);
+          rs4[i & 3] = add2(rs4[i & 3], pack2f(p0, p1));
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kKeys / 2; ++i) {
+          const uint64_t t2 = fma2(pack2(sv[2 * i], sv[2 * i + 1]), c2, off2);
+          float p0, p1;
+          if ((i & 7) < kPolyOf8) {
+            exp2_poly2(t2, p0, p1);
+          } else {
+            float t0, t1;
+            unpack2(t2, t0, t1);
+            p0 = ex2f(t0);
+            p1 = ex2f(t1);
+          }
+          rs4[i & 3] = add2(rs4[i & 3], pack2f(p0, p1));
+          pk[i] = pack_bf16x2(p0, p1);
+        }
       }
-      const float rowsum = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
-      l = l * alpha + rowsum;
+      float r0, r1;
+      unpack2(add2(add2(rs4[0], rs4[1]), add2(rs4[2], rs4[3])), r0, r1);
+      l = l * alpha + (r0 + r1);
 
-      if (j > 0) {  // P and O are free once the previous tile's P V has completed
-        ok = ok && mbar_wait(bar(PV_DONE), (j - 1) & 1, abort_flag);
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        // rare: the exponent offset moved.  O must be at rest: wait for P V of tile j-1 (P V of
+        // tile j cannot start before this thread publishes P_j), then rescale the row.
+        ok = ok && mbar_wait(bar(PV_DONE + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {  // rare: the exponent offset moved, rescale O
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t ov[32];
-            TSD_TMEM_LD32(ov, 0, t_lane + 256 + q4 * 32);
-            tmem_wait_ld();
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t ov[32];
+          TSD_TMEM_LD32(ov, 0, t_lane + kColO + q4 * 32);
+          tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-            TSD_TMEM_ST32(ov, 0, t_lane + 256 + q4 * 32);
-          }
-          tmem_wait_st();
+          for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+          TSD_TMEM_ST32(ov, 0, t_lane + kColO + q4 * 32);
         }
       }
-      // P (bf16) into the 128B-swizzled K-major tile: row r, 16-byte chunk cc at position cc ^ (r & 7)
-      const uint32_t prow = base + kOffP + (uint32_t)r * 128u;
-#pragma unroll
-      for (int cc = 0; cc < 16; ++cc) {
-        const uint32_t addr = prow + (cc >> 3) * kSub + (((uint32_t)(cc & 7) ^ (uint32_t)(r & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * cc]), "r"(pk[4 * cc + 1]),
-                     "r"(pk[4 * cc + 2]), "r"(pk[4 * cc + 3]) : "memory");
-      }
-      fence_async_smem();
+      // P (bf16 pairs) over the first 32 columns of this S buffer: column i = keys 2i (low half), 2i+1
+      TSD_TMEM_ST32(pk, 0, t_s);
+      tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(P_FULL));
+      if (lane == 0) mbar_arrive(bar(P_FULL + b));
     }
     // epilogue: O / l -> bf16 -> global, lse
-    if (ok && T > 0) ok = mbar_wait(bar(PV_DONE), (T - 1) & 1, abort_flag);
+    if (ok && T > 0) ok = mbar_wait(bar(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag);
     if (ok) {
       tc_fence_after();
       const int i = qt * kTile + r;
@@ -380,7 +526,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t ov[32];
         if (T > 0) {
-          TSD_TMEM_LD32(ov, 0, t_lane + 256 + q4 * 32);
+          TSD_TMEM_LD32(ov, 0, t_lane + kColO + q4 * 32);
           tmem_wait_ld();
         } else {
 #pragma unroll
@@ -407,7 +553,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   __syncthreads();
   if (warp == 5) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
   }
   if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, TSD_STATUS_TIMEOUT);
 }
@@ -430,8 +576,9 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [S, rows, H, 128] bf16 with element strides (sb, sr, sh): box = 128 rows x 64 elements, 128B swizzle.
-static bool make_map(CUtensorMap* m, const void* ptr, int S, int rows, int H, int64_t sb, int64_t sr, int64_t sh) {
+// [S, rows, H, 128] bf16 with element strides (sb, sr, sh): box = box_rows x 64 elements, 128B swizzle.
+static bool make_map(CUtensorMap* m, const void* ptr, int S, int rows, int H, int64_t sb, int64_t sr, int64_t sh,
+                     int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn || rows < 1) return false;
   cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)rows, (cuuint64_t)S};
@@ -439,7 +586,7 @@ static bool make_map(CUtensorMap* m, const void* ptr, int S, int rows, int H, in
   // a size-1 dimension may carry any stride; give it a harmless valid one
   if (H == 1) strides[0] = 256;
   if (S == 1) strides[2] = strides[1] * (cuuint64_t)rows;
-  cuuint32_t box[4] = {64, 1, 128, 1};
+  cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -468,12 +615,12 @@ int launch_attention_tc(const AttnArgs& a) {
   const tsd_layout& L = a.L;
   const int N = L.n_branches * L.rows_per_branch;
   CUtensorMap mq, mkc, mvc, mkd, mvd;
-  bool ok = make_map(&mq, a.q, L.batch, N, L.n_q_heads, a.qs_b, a.qs_r, a.qs_h) &&
-            make_map(&mkd, a.kd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h) &&
-            make_map(&mvd, a.vd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h);
+  bool ok = make_map(&mq, a.q, L.batch, N, L.n_q_heads, a.qs_b, a.qs_r, a.qs_h, kTile) &&
+            make_map(&mkd, a.kd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h, kKeys) &&
+            make_map(&mvd, a.vd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h, kKeys);
   if (ok && L.n_cache > 0) {
-    ok = make_map(&mkc, a.kc, L.batch, L.n_cache, L.n_kv_heads, a.cs_b, a.cs_r, a.cs_h) &&
-         make_map(&mvc, a.vc, L.batch, L.n_cache, L.n_kv_heads, a.cs_b, a.cs_r, a.cs_h);
+    ok = make_map(&mkc, a.kc, L.batch, L.n_cache, L.n_kv_heads, a.cs_b, a.cs_r, a.cs_h, kKeys) &&
+         make_map(&mvc, a.vc, L.batch, L.n_cache, L.n_kv_heads, a.cs_b, a.cs_r, a.cs_h, kKeys);
   } else if (ok) {  // no cache: the cached maps are never dereferenced
     mkc = mkd;
     mvc = mvd;
