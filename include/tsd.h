@@ -172,6 +172,35 @@ int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32
                         uint32_t* status, tsd_stream_t stream);
 
 /* ---------------------------------------------------------------------------
+ * Stage 2 without a caller workspace (no counterpart in the paper: an interface
+ * convenience of this library).  Same computation and outputs as
+ * tsd_confidence_topk, for callers that cannot obtain device memory at call
+ * time: a server plug-in whose device pool is fixed at start-up, a decode loop
+ * that may not call cudaMalloc because it would stall the device mid-step.
+ * The per-segment partial results and per-row tickets go to a 1 MiB array that
+ * is part of the library image (every GPU that loads the library holds it
+ * until the process exits); tsd_confidence_topk_static_capacity() returns that
+ * size.  The call itself allocates and frees nothing.
+ *   - A shape whose scratch need exceeds the capacity is rejected with
+ *     TSD_ERR_WORKSPACE and nothing is launched; compare
+ *     tsd_confidence_topk_workspace_bytes() with the capacity beforehand, and
+ *     fall back to tsd_confidence_topk with your own workspace.
+ *   - The first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress, with that device current).  Make that first call
+ *     before any stream capture begins.
+ *   - All calls on a device share the one array, and it keeps whatever the
+ *     previous call left: each call re-zeroes the ticket words it uses (on
+ *     `stream`, ahead of its kernel) and overwrites the partial slots it reads.
+ *     Two calls that overlap on the GPU (different streams, no ordering) would
+ *     race on it: order them on one stream or with events.
+ * Arguments as for tsd_confidence_topk, minus the workspace.
+ * ------------------------------------------------------------------------- */
+size_t tsd_confidence_topk_static_capacity(void);
+int tsd_confidence_topk_static(const void* logits, int32_t dtype, int64_t n_rows, int32_t vocab,
+                               int64_t row_stride, int32_t k, float* conf, int32_t* topk_idx,
+                               float* topk_prob, float* lse, uint32_t* status, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
  * Stage 3 — acceptance (Section 3.3 "Verification procedure"; Alg. 1 Phase 1
  * for the high/low confidence split; Eqs. 6-7 for the top-1 fallback).
  * Per node p the decode rule U(p) is what threshold decoding would unmask

@@ -25,6 +25,7 @@ EXPORTS = (
     "tsd_branch_mask_bytes", "tsd_build_branch_mask",
     "tsd_verify_attention_workspace_bytes", "tsd_verify_attention",
     "tsd_confidence_topk_workspace_bytes", "tsd_confidence_topk",
+    "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
     "tsd_accept_trajectories",
 )
 
@@ -73,6 +74,9 @@ def lib():
         L.tsd_confidence_topk_workspace_bytes.argtypes = [_i64, _i32, _i32]
         L.tsd_confidence_topk.argtypes = [_vp, _i32, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
                                           _sz, _vp, _vp]
+        L.tsd_confidence_topk_static_capacity.restype = _sz
+        L.tsd_confidence_topk_static_capacity.argtypes = []
+        L.tsd_confidence_topk_static.argtypes = [_vp, _i32, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
         L.tsd_accept_trajectories.argtypes = [_i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
                                               _i32, _i32] + [_vp] * 9
         _lib = L
@@ -168,6 +172,20 @@ def tsd_confidence_topk(logits, k, conf, topk_idx, topk_prob, lse=None, workspac
         int(k), _ptr(conf), _ptr(topk_idx), _ptr(topk_prob), _ptr(lse), _ptr(workspace), ws_bytes,
         _ptr(status), _stream(stream))
     _check(rc, "tsd_confidence_topk")
+
+
+def tsd_confidence_topk_static_capacity():
+    return int(lib().tsd_confidence_topk_static_capacity())
+
+
+def tsd_confidence_topk_static(logits, k, conf, topk_idx, topk_prob, lse=None, status=None, stream=None):
+    """tsd_confidence_topk for callers that cannot provide a workspace: the scratch is the fixed
+    array inside the library (see the header for its limit and sharing rules)."""
+    assert logits.dim() == 2 and logits.stride(1) == 1
+    rc = lib().tsd_confidence_topk_static(
+        _ptr(logits), dtype_code(logits.dtype), logits.shape[0], logits.shape[1], logits.stride(0),
+        int(k), _ptr(conf), _ptr(topk_idx), _ptr(topk_prob), _ptr(lse), _ptr(status), _stream(stream))
+    _check(rc, "tsd_confidence_topk_static")
 
 
 def tsd_accept_trajectories(parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule, search,

@@ -22,6 +22,7 @@
 #include <limits.h>
 #include <math_constants.h>
 #include <algorithm>
+#include <mutex>
 #include "tsd_common.cuh"
 
 namespace tsd {
@@ -492,3 +493,74 @@ int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant.  Some hosts can hand this library nothing but their inputs and outputs:
+// an inference-server plug-in whose device memory pool is sized once at start-up and then frozen,
+// or a decode loop in which calling cudaMalloc is ruled out because it would stall the whole
+// device in the middle of a step.  For them the per-segment partial results and the per-row
+// tickets live in a fixed array that is part of the library image: every GPU that loads the
+// library carries these bytes until the process exits, which is why the size is kept modest.
+namespace tsd {
+
+constexpr size_t kStaticScratchBytes = 1u << 20;  // 1 MiB per device
+static __device__ __align__(256) unsigned char g_topk_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mutex;
+static void* g_scratch_ptr[kMaxDevices] = {};  // device address of g_topk_scratch, per device
+
+// In host code `g_topk_scratch` is only a handle for the runtime, not an address a kernel can use:
+// the device address has to be asked for, once per device, with that device current.
+static cudaError_t static_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_topk_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_ptr[dev] = ptr;
+  }
+  *out = g_scratch_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace tsd
+
+extern "C" size_t tsd_confidence_topk_static_capacity(void) { return tsd::kStaticScratchBytes; }
+
+extern "C" int tsd_confidence_topk_static(const void* logits, int32_t dtype, int64_t n_rows, int32_t vocab,
+                                          int64_t row_stride, int32_t k, float* conf, int32_t* topk_idx,
+                                          float* topk_prob, float* lse, uint32_t* status,
+                                          tsd_stream_t stream) {
+  (void)status;
+  int rc = topk_check(n_rows, vocab, k);
+  if (rc != TSD_OK) return rc;
+  if (dtype != TSD_F32 && dtype != TSD_BF16) return TSD_ERR_UNSUPPORTED;
+  if (n_rows == 0) return TSD_OK;
+  const int esize = dtype == TSD_F32 ? 4 : 2;
+  if (!logits || !conf || !topk_idx || !topk_prob) return TSD_ERR_INVALID_ARG;
+  if (row_stride < vocab || !tsd::aligned16(logits) || (row_stride * esize) % 16 != 0)
+    return TSD_ERR_INVALID_ARG;
+  const tsd::TopkPlan p = tsd::topk_plan(n_rows, vocab, k, 16 / esize);
+  // this shape would need more scratch than the library carries: the caller has to use
+  // tsd_confidence_topk with a workspace of its own
+  if (p.total_bytes > tsd::kStaticScratchBytes) return TSD_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  if (p.total_bytes > 0) {
+    cudaError_t e = tsd::static_scratch_address(&scratch);
+    if (e != cudaSuccess) return tsd::cuda_fail(e, "cudaGetSymbolAddress(g_topk_scratch)");
+  }
+  // the launcher zeroes the ticket words inside the scratch on the stream before the kernel; the
+  // partial-result slots are fully rewritten by every call that reads them
+  cudaError_t e = dtype == TSD_F32
+      ? tsd::dispatch_k<float>(p.K, logits, n_rows, vocab, row_stride, k, p, conf, topk_idx, topk_prob,
+                               lse, scratch, stream)
+      : tsd::dispatch_k<__nv_bfloat16>(p.K, logits, n_rows, vocab, row_stride, k, p, conf, topk_idx,
+                                       topk_prob, lse, scratch, stream);
+  if (e != cudaSuccess) return tsd::cuda_fail(e, "confidence_topk_kernel (static scratch)");
+  return TSD_OK;
+}
