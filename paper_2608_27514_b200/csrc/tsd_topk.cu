@@ -27,11 +27,8 @@
 
 namespace tsd {
 
-constexpr int kTopkThreads = 256;
-constexpr int kTopkWarps = kTopkThreads / 32;
-constexpr int kTopkUnroll = 4;                          // chunks per thread per batch
-constexpr int kTopkBatch = kTopkThreads * kTopkUnroll;  // chunks per block per batch
-constexpr int kTopkMaxIter = 32;                        // batches per segment (batch maxima kept in smem)
+constexpr int kTopkUnroll = 4;            // chunks per thread per batch
+constexpr int kTopkSegChunks = 32768;     // chunks per segment at most (batch maxima: 32 KB of smem)
 constexpr int kMaxSegments = 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -225,14 +222,18 @@ struct Unpack<__nv_bfloat16> {
   }
 };
 
-// grid.x = n_rows * n_seg; block = kTopkThreads.
-template <typename T, int K>
-__global__ void __launch_bounds__(kTopkThreads)
+// grid.x = n_rows * n_seg; block = THREADS (256 when many blocks share an SM; 512 when there are so
+// few rows that a block has to keep the SM busy on its own: twice the warps per row).
+template <typename T, int K, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stride, int k, int n_seg,
                        int chunks_per_seg, float* __restrict__ conf, int32_t* __restrict__ topk_idx,
                        float* __restrict__ topk_prob, float* __restrict__ lse,
                        Partial<K>* __restrict__ partials, unsigned* __restrict__ tickets) {
   constexpr int E = Unpack<T>::kElems;
+  constexpr int kTopkThreads = THREADS, kTopkWarps = THREADS / 32;
+  constexpr int kTopkBatch = THREADS * kTopkUnroll;        // chunks per block per batch
+  constexpr int kTopkMaxIter = kTopkSegChunks / kTopkBatch;  // batches per segment
   __shared__ float s_bmax[kTopkMaxIter][kTopkThreads];  // per-thread batch maxima
   __shared__ float s_top[kTopkWarps][K];
   __shared__ Partial<K> s_part[kTopkWarps];
@@ -247,11 +248,11 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   const int n_iter = (c1 - c0 + kTopkBatch - 1) / kTopkBatch;  // <= kTopkMaxIter (host-enforced)
   const bool has_tail = seg == n_seg - 1 && tid == 0 && chunks_total * E < vocab;
 
-  // ---- phase 1: stream
+  // ---- phase 1: stream.  Two register buffers: the loads of batch it+1 are in flight while
+  // batch it is processed, so a block overlaps memory latency with its own arithmetic.
   float m = -CUDART_INF_F, e = 0.f, s = 0.f;
-  for (int it = 0; it < n_iter; ++it) {
+  auto load_batch = [&](uint4 (&buf)[kTopkUnroll], int it) {
     const int base = c0 + it * kTopkBatch + tid;
-    uint4 buf[kTopkUnroll];
 #pragma unroll
     for (int u = 0; u < kTopkUnroll; ++u) {
       const int c = base + u * kTopkThreads;
@@ -260,6 +261,8 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
         buf[u] = make_uint4(Unpack<T>::kNegInfWord, Unpack<T>::kNegInfWord, Unpack<T>::kNegInfWord,
                             Unpack<T>::kNegInfWord);
     }
+  };
+  auto process_batch = [&](const uint4 (&buf)[kTopkUnroll], int it) {
     const float bm = Unpack<T>::batch_max(buf);
     s_bmax[it][tid] = bm;
     const float m_new = fmaxf(m, bm);
@@ -267,8 +270,22 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     s *= (m == -CUDART_INF_F) ? 0.f : ex2_approx(e - e_new);  // rebase: 1 when the maximum stays
     m = m_new;
     e = e_new;
+    float part[kTopkUnroll];  // independent partial sums keep the dependent add chains short
 #pragma unroll
-    for (int u = 0; u < kTopkUnroll; ++u) s = Unpack<T>::sum_exp(buf[u], -e, s);
+    for (int u = 0; u < kTopkUnroll; ++u) part[u] = Unpack<T>::sum_exp(buf[u], -e, 0.f);
+    s += (part[0] + part[1]) + (part[2] + part[3]);
+  };
+  {
+    uint4 buf_a[kTopkUnroll], buf_b[kTopkUnroll];
+    if (n_iter > 0) load_batch(buf_a, 0);
+    for (int it = 0; it < n_iter; it += 2) {
+      if (it + 1 < n_iter) load_batch(buf_b, it + 1);
+      process_batch(buf_a, it);
+      if (it + 1 < n_iter) {
+        if (it + 2 < n_iter) load_batch(buf_a, it + 2);
+        process_batch(buf_b, it + 1);
+      }
+    }
   }
   float tail_max = -CUDART_INF_F;
   if (has_tail) {  // ragged tail of a vocabulary that is not a multiple of the chunk size
@@ -290,19 +307,26 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   }
   __syncthreads();
   {
-    // every warp redoes the small cross-warp step: lanes hold the 8 x K warp values
-    float x = -CUDART_INF_F, bound = -CUDART_INF_F;
-    // K rounds over up to 32 candidate values per round-robin slice (8*K <= 64)
-    float c0v = lane < kTopkWarps * K ? s_top[lane / K][lane % K] : -CUDART_INF_F;
-    float c1v = lane + 32 < kTopkWarps * K ? s_top[(lane + 32) / K][(lane + 32) % K] : -CUDART_INF_F;
+    // every warp redoes the small cross-warp step: the lanes hold the WARPS x K warp values
+    constexpr int NV = (kTopkWarps * K + 31) / 32;
+    float cv[NV];
+#pragma unroll
+    for (int q = 0; q < NV; ++q) {
+      const int idx = lane + 32 * q;
+      cv[q] = idx < kTopkWarps * K ? s_top[idx / K][idx % K] : -CUDART_INF_F;
+    }
+    float bound = -CUDART_INF_F;
 #pragma unroll
     for (int r = 0; r < K; ++r) {
-      x = fmaxf(c0v, c1v);
+      float x = cv[0];
+#pragma unroll
+      for (int q = 1; q < NV; ++q) x = fmaxf(x, cv[q]);
 #pragma unroll
       for (int off = 16; off; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, off));
       bound = x;
-      if (c0v == x) c0v = -CUDART_INF_F;
-      if (c1v == x) c1v = -CUDART_INF_F;
+#pragma unroll
+      for (int q = 0; q < NV; ++q)
+        if (cv[q] == x) cv[q] = -CUDART_INF_F;
     }
     top[0] = bound;
   }
@@ -386,7 +410,7 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
 }
 
 struct TopkPlan {
-  int n_seg, chunks_per_seg, K;
+  int n_seg, chunks_per_seg, K, threads;
   size_t partial_bytes, ticket_off, total_bytes;
 };
 
@@ -396,14 +420,17 @@ static TopkPlan topk_plan(int64_t n_rows, int vocab, int k, int elems_per_chunk)
   TopkPlan p;
   p.K = round_k(k);
   const int chunks = vocab / elems_per_chunk;
-  const int64_t target_units = 148 * 16;
+  // Few rows: split rows only until every SM has a block (more segments add per-block latency
+  // and merge work faster than they add parallelism; measured on cfg2- and cfg3-sized inputs).
+  const int64_t target_units = 148;
   int64_t n_seg = n_rows >= target_units ? 1 : (target_units + n_rows - 1) / n_rows;
   n_seg = std::min<int64_t>(n_seg, kMaxSegments);
-  n_seg = std::min<int64_t>(n_seg, std::max(1, chunks / 1024));
-  // a segment may span at most kTopkMaxIter batches (its batch maxima live in shared memory)
-  const int64_t seg_cap = (int64_t)kTopkBatch * kTopkMaxIter;
-  n_seg = std::max<int64_t>(n_seg, (chunks + seg_cap - 1) / seg_cap);
+  n_seg = std::min<int64_t>(n_seg, std::max(1, chunks / 2048));
+  // a segment may span at most kTopkSegChunks chunks (its batch maxima live in shared memory)
+  n_seg = std::max<int64_t>(n_seg, (chunks + kTopkSegChunks - 1) / kTopkSegChunks);
   p.n_seg = (int)std::max<int64_t>(n_seg, 1);
+  // up to two 512-thread blocks fit an SM: use them while that still gives every block a slot at once
+  p.threads = (n_rows * p.n_seg <= 2 * 148) ? 512 : 256;
   p.chunks_per_seg = (chunks + p.n_seg - 1) / p.n_seg;
   if (p.chunks_per_seg == 0) p.chunks_per_seg = 1;
   const size_t rec = 8 + 8 * (size_t)p.K;
@@ -423,9 +450,14 @@ static cudaError_t launch_topk(const void* logits, int64_t n_rows, int vocab, in
     cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)n_rows * 4, st);
     if (e != cudaSuccess) return e;
   }
-  confidence_topk_kernel<T, K><<<(unsigned)(n_rows * p.n_seg), kTopkThreads, 0, st>>>(
-      static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
-      lse, partials, tickets);
+  if (p.threads == 512)
+    confidence_topk_kernel<T, K, 512><<<(unsigned)(n_rows * p.n_seg), 512, 0, st>>>(
+        static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
+        lse, partials, tickets);
+  else
+    confidence_topk_kernel<T, K, 256><<<(unsigned)(n_rows * p.n_seg), 256, 0, st>>>(
+        static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
+        lse, partials, tickets);
   return cudaGetLastError();
 }
 
@@ -451,7 +483,7 @@ static int topk_check(int64_t n_rows, int32_t vocab, int32_t k) {
   if (n_rows < 0 || vocab < 1 || k < 1 || k > 8 || k > vocab) return TSD_ERR_INVALID_ARG;
   if (n_rows * (int64_t)tsd::kMaxSegments > 0x7fffffffLL) return TSD_ERR_INVALID_ARG;
   // rows longer than kMaxSegments segments of kTopkMaxIter batches (4 Mi fp32 / 8 Mi bf16 logits)
-  if ((int64_t)vocab / 4 > (int64_t)tsd::kTopkBatch * tsd::kTopkMaxIter * tsd::kMaxSegments)
+  if ((int64_t)vocab / 4 > (int64_t)tsd::kTopkSegChunks * tsd::kMaxSegments)
     return TSD_ERR_INVALID_ARG;
   return TSD_OK;
 }

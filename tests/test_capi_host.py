@@ -65,7 +65,7 @@ def test_topk_validation(lib):
     assert call(logits=ctypes.c_void_p(4098)) == B.TSD_ERR_INVALID_ARG
     assert call(stride=1020) == B.TSD_ERR_INVALID_ARG          # shorter than the vocabulary
     assert call(vocab=1000, stride=1004) == B.TSD_ERR_INVALID_ARG  # row pitch not a 16-byte multiple
-    need = B.tsd_confidence_topk_workspace_bytes(4, 126464, 3)
+    need = B.tsd_confidence_topk_workspace_bytes(4, 126464, 3)   # few rows: rows are split into segments
     assert need > 0
     assert call(vocab=126464, stride=126464, ws_bytes=need - 1) == B.TSD_ERR_WORKSPACE
     assert call(vocab=126464, stride=126464, ws=None) == B.TSD_ERR_INVALID_ARG
