@@ -62,6 +62,13 @@ def algorithmic(cfg):
     return dict(attn_flops=attn_flops, attn_bytes=attn_bytes, topk_bytes=topk_bytes)
 
 
+def base_config(cfg, world=1):
+    """The workload description both arms report."""
+    return dict(workload=cfg.name, batch=cfg.S, branches=cfg.B, rows_per_branch=cfg.R, rows=cfg.rows,
+                n_cache=cfg.Nc, q_heads=cfg.Hq, kv_heads=cfg.Hkv, head_dim=cfg.d, vocab=cfg.V, k=cfg.k,
+                tau=cfg.tau, attention_layers_per_step=1, parallelism="replicas" if world > 1 else "1gpu")
+
+
 class ClockSampler:
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -183,7 +190,7 @@ def run_reference(args, cfg):
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
-                config=dict(workload=cfg.name, rows=cfg.rows, note="CPU oracle, fp64, sampled and scaled"),
+                config=dict(base_config(cfg), note="CPU oracle, fp64, bounded sample scaled to the full step"),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle",
                                   sample=last["sample"]),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
@@ -214,17 +221,14 @@ def main():
     from paper_2608_27514_b200 import binding as B
     from paper_2608_27514_b200.step import VerifyStep
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2608_27514_b200 import replicas
+    rank, local_rank, world = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     B.lib()  # fail loudly if the CUDA library is missing
     torch.cuda.set_device(local_rank)
     dev = "cuda:%d" % local_rank
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    replicas.init("nccl", dev)
 
     alg = algorithmic(cfg)
     pk = peaks()
@@ -272,9 +276,7 @@ def main():
             run_step(i)
 
     def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     # ---------------- timed region A: K whole steps, inputs resident in HBM
@@ -373,11 +375,7 @@ def main():
     e2e_ms = max(a.elapsed_time(b), (time.perf_counter() - t0) * 1e3) / e2e_steps
 
     # ---------------- reduce over ranks (replicas: the slowest rank sets the time)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_ms = float(t[0]), float(t[1])
+    elapsed_ms, e2e_ms = replicas.max_over_ranks([elapsed_ms, e2e_ms], dev)
     ms_per_step = elapsed_ms / args.steps
     value = world * cfg.rows / (ms_per_step * 1e-3)
 
@@ -410,9 +408,7 @@ def main():
                     algorithmic_bytes=alg["attn_bytes"], peak_source=pk["source"])
 
     if rank != 0:
-        if world > 1:
-            import torch.distributed as dist
-            dist.destroy_process_group()
+        replicas.shutdown()
         return
 
     cpu = None
@@ -426,9 +422,7 @@ def main():
         metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
-        config=dict(workload=cfg.name, batch=cfg.S, branches=cfg.B, rows_per_branch=cfg.R, rows=cfg.rows,
-                    n_cache=cfg.Nc, q_heads=cfg.Hq, kv_heads=cfg.Hkv, head_dim=cfg.d, vocab=cfg.V, k=cfg.k,
-                    tau=cfg.tau, attention_layers_per_step=1, parallelism="replicas" if world > 1 else "1gpu",
+        config=dict(base_config(cfg, world),
                     l2_hygiene=("inputs larger than L2" if n_copies == 1 else
                                 "rotating %d input copies (%.0f MB total, L2 is 126 MB)"
                                 % (n_copies, n_copies * in_bytes / 1e6)),
@@ -439,9 +433,7 @@ def main():
         gpu_launches=launches_per_step * args.steps,
         roofline=roof, stages=stages, cpu_baseline=cpu)
     print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 if __name__ == "__main__":
