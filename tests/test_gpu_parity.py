@@ -357,3 +357,59 @@ def test_topk_subnormal_and_signed_zero_logits():
     x[3, :] = -tiny
     x[3, 9], x[3, 10] = -0.0, 0.0
     _check_topk(x, 4)
+
+
+# ------------------------------------------------------------------------ extremes
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_many_branches_all_visible(flags):
+    # 256 branches (the maximum) that all see each other: every query tile lists all 64 draft tiles
+    cfg = W.small(W.CONFIGS["cfg2"], B=256, R=32, Nc=64, Hq=1, Hkv=1)
+    vis = torch.full((cfg.S, cfg.B, 4), -1, dtype=torch.int64, device=DEV)
+    _check_attention(cfg, W.attention_inputs(cfg, DEV), flags, vis=vis)
+
+
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_batch_with_an_empty_cache(flags):
+    # one sequence of the batch has no valid cached token at all: only its own branch is visible
+    cfg = W.small(W.CONFIGS["cfg2"], S=3, B=4, R=64, Nc=200, Hq=2, Hkv=1)
+    lens = torch.tensor([200, 0, 1], dtype=torch.int32, device=DEV)
+    _check_attention(cfg, W.attention_inputs(cfg, DEV), flags, cache_lens=lens)
+
+
+def test_topk_k_equals_vocab_and_single_row():
+    g = torch.Generator(device=DEV).manual_seed(9)
+    x = torch.randn((5, 8), generator=g, device=DEV).bfloat16()
+    _check_topk(x, 8)                                  # every entry is a candidate
+    y = torch.randn((1, 300000), generator=g, device=DEV)
+    _check_topk(y, 8)                                  # one long fp32 row: segments + ticket merge
+    z = torch.randn((3, 16), generator=g, device=DEV)
+    _check_topk(z[:, :1], 1)                           # vocabulary of one
+
+
+def test_accept_largest_tree():
+    rng = np.random.default_rng(3)
+    S, Bn, R, V = 2, 256, 128, 1000
+    M = V
+    parent = np.stack([[-1] + [int(rng.integers(max(0, b - 3), b)) for b in range(1, Bn)] for _ in range(S)]).astype(np.int32)
+    conf = rng.random((S, Bn, R)).astype(np.float32)
+    top1 = rng.integers(0, V, (S, Bn, R)).astype(np.int32)
+    state = np.full((S, Bn, R), M, np.int32)
+    for s in range(S):
+        for b in range(1, Bn):
+            p = parent[s, b]
+            c = state[s, p].copy()
+            flag, tok = oracle.decode_rule(state[s, p], M, conf[s, p], top1[s, p], 0.97)
+            if rng.random() < 0.8:
+                c[flag.astype(bool)] = tok[flag.astype(bool)]
+            else:
+                rows = np.flatnonzero(c == M)
+                if len(rows):
+                    c[rows[-1]] = rng.integers(0, V)
+            state[s, b] = c
+    for rule in (0, 1):
+        for search in (0, 1):
+            ref = oracle.accept(parent, state, M, conf, top1, 0.97, rule, search)
+            got, status = _gpu_accept(parent, state, M, conf, top1, 0.97, rule, search)
+            for key, val in ref.items():
+                assert np.array_equal(got[key], val), (key, rule, search)
+            assert ref["accepted_len"].max() > 3          # deep chains really are accepted
