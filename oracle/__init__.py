@@ -15,4 +15,5 @@ from .binding import (  # noqa: F401
     confidence_topk,
     decode_rule,
     accept,
+    build_draft_tree,
 )

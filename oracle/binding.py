@@ -135,3 +135,21 @@ def accept(parent, state, mask_id, conf, top1, tau, rule=0, search=0):
         _ptr(o["accepted_len"]), _ptr(o["n_new_tokens"]), _ptr(o["unmask_flag"]),
         _ptr(o["unmask_tok"]))
     return o
+
+
+def build_draft_tree(root_state, mask_id, topk_idx, topk_prob, W, D, max_nodes):
+    """One sequence: root_state [R], topk_idx/topk_prob [R,k] -> (n_nodes, parent [B], state [B,R],
+    node_prob [B]) by Alg. 1 Phase 2 (see the C source for the reading of its three helpers)."""
+    root_state = _arr(root_state, np.int32)
+    topk_idx = _arr(topk_idx, np.int32)
+    topk_prob = _arr(topk_prob, np.float32)
+    R, k = topk_idx.shape
+    parent = np.empty(max_nodes, np.int32)
+    state = np.empty((max_nodes, R), np.int32)
+    prob = np.empty(max_nodes, np.float32)
+    lib = _load()
+    lib.oracle_build_draft_tree.restype = ctypes.c_int
+    n = lib.oracle_build_draft_tree(R, k, _ptr(root_state), ctypes.c_int32(mask_id), _ptr(topk_idx),
+                                    _ptr(topk_prob), int(W), int(D), int(max_nodes), _ptr(parent),
+                                    _ptr(state), _ptr(prob))
+    return int(n), parent, state, prob

@@ -97,6 +97,10 @@ def _draft(model, root, conf, idx, prob, mode, rng, tau, peek):
 
     if not masked:
         return np.stack(nodes), parent
+    if mode == "alg1":
+        # the library's reading of Alg. 1 Phase 2 on the previous pass's candidate pool (W2D2(3))
+        n, par, st, _ = _o.build_draft_tree(root, model.mask_id, idx, prob.astype(np.float32), 2, 2, 4)
+        return st[:n].astype(np.int32), [int(x) for x in par[:n]]
     if mode == "peek":
         steps = peek[:3]
         wrong_r = masked[int(rng.integers(len(masked)))]

@@ -17,6 +17,7 @@
  *   oracle_decode_rule       Alg. 1 Phase 1 (H = {conf > tau}) with the top-1
  *                            fallback of Eqs. 6-7
  *   oracle_accept            Section 3.3 "Verification procedure" (greedy / longest path)
+ *   oracle_build_draft_tree  Alg. 1 Phase 2 (the step before the path; built after it)
  *
  * Pins (tests/test_oracle_*.py): textbook attention for one branch, plain
  * bidirectional attention for an all-visible mask, per-row brute force,
@@ -322,4 +323,102 @@ void oracle_accept(int S, int B, int R, const int32_t* parent,
   free(utok);
   free(t1);
   free(depth);
+}
+
+/* ------------------------------------------------------------------------
+ * Alg. 1, Phase 2 (speculative expansion) for one sequence.  The root block
+ * state is given (Phase 1, filling the rows above tau, is what the caller
+ * does with the previous step's unmask set); the candidate pool of Section 3.2
+ * is the top-k (token, probability) of every row that is still masked in the
+ * root, taken from the scores of the previous verification pass.
+ *
+ * The paper names but does not define GenerateTopK, GenerateTop1 and
+ * PruneByConfidence; the reading implemented here:
+ *   level 1  (GenerateTopK): the k best pool entries (row, j) by probability
+ *            (ties: lower row, then lower rank j), one child per entry =
+ *            root + that one (row, token);
+ *   level >1 (GenerateTop1): every frontier node gets one child = the node +
+ *            the best pool entry whose row is still masked in that node;
+ *   PruneByConfidence: keep the W children of a level whose added entry has
+ *            the largest probability (ties: earlier in generation order), in
+ *            that order; they become the next frontier;
+ *   the tree holds at most max_nodes nodes (the "n child blocks" of the
+ *   WxDy(n) naming, plus the root): a level is cut where the budget ends.
+ * Nodes are numbered level by level in pruned order, so siblings are listed in
+ * descending draft confidence.  Unused node slots are copies of the root with
+ * parent 0 (an empty delta: never valid).
+ * Outputs: parent[max_nodes], state[max_nodes][R], node_prob[max_nodes]
+ * (probability of the entry the node added; root: 1), returns the node count.
+ * ---------------------------------------------------------------------- */
+int oracle_build_draft_tree(int R, int k, const int32_t* root_state, int32_t mask_id,
+                            const int32_t* topk_idx, const float* topk_prob, int W, int D,
+                            int max_nodes, int32_t* parent, int32_t* state, float* node_prob) {
+  int n = 1;
+  parent[0] = -1;
+  node_prob[0] = 1.0f;
+  memcpy(state, root_state, sizeof(int32_t) * (size_t)R);
+  for (int b = 1; b < max_nodes; ++b) {
+    parent[b] = 0;
+    node_prob[b] = 0.0f;
+    memcpy(state + (size_t)b * R, root_state, sizeof(int32_t) * (size_t)R);
+  }
+  int* frontier = (int*)malloc(sizeof(int) * (size_t)(max_nodes > 0 ? max_nodes : 1));
+  int n_front = 1;
+  frontier[0] = 0;
+  /* children of one level before pruning: (parent node, row, rank) */
+  const int cap = (k > max_nodes ? k : max_nodes) + 1;
+  int* c_par = (int*)malloc(sizeof(int) * (size_t)cap);
+  int* c_row = (int*)malloc(sizeof(int) * (size_t)cap);
+  int* c_rank = (int*)malloc(sizeof(int) * (size_t)cap);
+  uint8_t* used = (uint8_t*)malloc((size_t)R * (size_t)k);
+  for (int level = 1; level <= D && n < max_nodes && n_front > 0; ++level) {
+    int n_child = 0;
+    if (level == 1) {
+      memset(used, 0, (size_t)R * (size_t)k);
+      for (int t = 0; t < k; ++t) {  /* the k best pool entries, one scan each */
+        int br = -1, bj = -1;
+        for (int r = 0; r < R; ++r) {
+          if (root_state[r] != mask_id) continue;
+          for (int j = 0; j < k; ++j) {
+            if (used[r * k + j]) continue;
+            if (br < 0 || topk_prob[r * k + j] > topk_prob[br * k + bj]) { br = r; bj = j; }
+          }
+        }
+        if (br < 0) break;
+        used[br * k + bj] = 1;
+        c_par[n_child] = 0; c_row[n_child] = br; c_rank[n_child] = bj; ++n_child;
+      }
+    } else {
+      for (int f = 0; f < n_front; ++f) {
+        const int32_t* ps = state + (size_t)frontier[f] * R;
+        int br = -1, bj = -1;
+        for (int r = 0; r < R; ++r) {
+          if (ps[r] != mask_id) continue;
+          for (int j = 0; j < k; ++j)
+            if (br < 0 || topk_prob[r * k + j] > topk_prob[br * k + bj]) { br = r; bj = j; }
+        }
+        if (br < 0) continue;  /* the node is full: nothing left to speculate on */
+        c_par[n_child] = frontier[f]; c_row[n_child] = br; c_rank[n_child] = bj; ++n_child;
+      }
+    }
+    /* PruneByConfidence: stable selection of the W most probable children */
+    n_front = 0;
+    for (int w = 0; w < W && n < max_nodes; ++w) {
+      int best = -1;
+      for (int c = 0; c < n_child; ++c) {
+        if (c_par[c] < 0) continue;
+        if (best < 0 || topk_prob[c_row[c] * k + c_rank[c]] > topk_prob[c_row[best] * k + c_rank[best]]) best = c;
+      }
+      if (best < 0) break;
+      const int b = n++;
+      parent[b] = c_par[best];
+      memcpy(state + (size_t)b * R, state + (size_t)c_par[best] * R, sizeof(int32_t) * (size_t)R);
+      state[(size_t)b * R + c_row[best]] = topk_idx[c_row[best] * k + c_rank[best]];
+      node_prob[b] = topk_prob[c_row[best] * k + c_rank[best]];
+      frontier[n_front++] = b;
+      c_par[best] = -1;
+    }
+  }
+  free(frontier); free(c_par); free(c_row); free(c_rank); free(used);
+  return n;
 }
