@@ -232,6 +232,35 @@ int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_
                             int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
                             int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream);
 
+/* ---------------------------------------------------------------------------
+ * Draft-tree construction for the next step (Alg. 1 "Confidence-Stratified
+ * Trajectory Tree Construction", Phase 2; Section 3.2 hybrid expansion), fused
+ * with the root update after acceptance so that a decode step stays on the
+ * device.  Per sequence: next root = state of the accepted node + its unmask
+ * set; candidate pool = top-k (token, probability) of the rows still masked in
+ * that root, from the scores of the pass just verified (Section 3.1).
+ * Level 1: the k most probable pool entries, one child each; deeper levels: one
+ * child per frontier node (its most probable entry at a row it still masks);
+ * after each level the `width` most probable children survive (siblings end up
+ * in descending draft confidence); the tree holds at most `max_nodes` nodes
+ * (the WxDy(n) naming: n + 1).  Ties: lower row, lower rank, earlier child.
+ *
+ *   prev_state    device int32 [batch, prev_branches, R]: block states of the verified tree.
+ *   accepted_node device int32 [batch], nullable (= node 0).
+ *   unmask_flag, unmask_tok   device [batch, R], both or neither: U(accepted node).
+ *   topk_idx, topk_prob       device [batch, prev_branches, R, k]: stage 2 output of that pass.
+ *   parent        device int32 [batch, max_nodes];  state device int32 [batch, max_nodes, R];
+ *   node_prob     device fp32 [batch, max_nodes]: probability of the entry a node added (root 1);
+ *   n_nodes       device int32 [batch].  Slots past n_nodes are copies of the root with parent 0.
+ * R 1..128, k 1..8, width 1..32, depth >= 0, max_nodes 1..256.
+ * ------------------------------------------------------------------------- */
+int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_t rows_per_branch, int32_t k,
+                         const int32_t* prev_state, const int32_t* accepted_node,
+                         const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
+                         const int32_t* topk_idx, const float* topk_prob, int32_t width, int32_t depth,
+                         int32_t max_nodes, int32_t* parent, int32_t* state, float* node_prob,
+                         int32_t* n_nodes, uint32_t* status, tsd_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

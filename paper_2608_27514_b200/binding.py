@@ -26,7 +26,7 @@ EXPORTS = (
     "tsd_verify_attention_workspace_bytes", "tsd_verify_attention",
     "tsd_confidence_topk_workspace_bytes", "tsd_confidence_topk",
     "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
-    "tsd_accept_trajectories",
+    "tsd_accept_trajectories", "tsd_build_draft_tree",
 )
 
 
@@ -79,6 +79,8 @@ def lib():
         L.tsd_confidence_topk_static.argtypes = [_vp, _i32, _i64, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
         L.tsd_accept_trajectories.argtypes = [_i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
                                               _i32, _i32] + [_vp] * 9
+        L.tsd_build_draft_tree.argtypes = [_i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32,
+                                           _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
         _lib = L
     return _lib
 
@@ -198,3 +200,16 @@ def tsd_accept_trajectories(parent, state, mask_id, conf, top1_idx, top1_stride,
         _ptr(accepted_len), _ptr(n_new_tokens), _ptr(unmask_flag), _ptr(unmask_tok), _ptr(status),
         _stream(stream))
     _check(rc, "tsd_accept_trajectories")
+
+
+def tsd_build_draft_tree(prev_state, accepted_node, unmask_flag, unmask_tok, mask_id, topk_idx, topk_prob,
+                         width, depth, parent, state, node_prob, n_nodes, status=None, stream=None):
+    """prev_state [S,Bp,R]; topk_idx/topk_prob [S*Bp*R, k] (or any shape with that many entries);
+    outputs parent [S,B], state [S,B,R], node_prob [S,B], n_nodes [S]."""
+    S, Bp, R = prev_state.shape
+    k = topk_idx.shape[-1]
+    rc = lib().tsd_build_draft_tree(
+        S, Bp, R, k, _ptr(prev_state), _ptr(accepted_node), _ptr(unmask_flag), _ptr(unmask_tok), int(mask_id),
+        _ptr(topk_idx), _ptr(topk_prob), int(width), int(depth), int(state.shape[1]), _ptr(parent), _ptr(state),
+        _ptr(node_prob), _ptr(n_nodes), _ptr(status), _stream(stream))
+    _check(rc, "tsd_build_draft_tree")

@@ -115,3 +115,19 @@ def test_missing_library_is_loud(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libtsd.so")
     with pytest.raises(RuntimeError, match="no fallback"):
         B.lib()
+
+
+def test_tree_validation(lib):
+    p = ctypes.c_void_p(4096)
+    f = lib.tsd_build_draft_tree
+
+    def call(S=1, Bp=4, R=32, k=3, prev=p, flag=p, tok=p, W=2, D=2, B_=4):
+        return f(S, Bp, R, k, prev, p, flag, tok, 99, p, p, W, D, B_, p, p, p, p, None, None)
+    assert call(R=129) == B.TSD_ERR_INVALID_ARG
+    assert call(k=9) == B.TSD_ERR_INVALID_ARG
+    assert call(W=0) == B.TSD_ERR_INVALID_ARG
+    assert call(W=33) == B.TSD_ERR_INVALID_ARG
+    assert call(B_=257) == B.TSD_ERR_INVALID_ARG
+    assert call(flag=None) == B.TSD_ERR_INVALID_ARG      # flag without tokens
+    assert call(prev=None) == B.TSD_ERR_INVALID_ARG
+    assert call(S=0) == B.TSD_OK
