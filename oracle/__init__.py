@@ -5,7 +5,8 @@ paper's definitions in ``tsd_oracle.c`` and loaded here through ctypes.  Only
 tests, the smoke check and the benchmark's CPU-baseline leg may import this
 package; the CUDA library never does, and the two share no code.
 
-``theorem1`` holds the toy-model harness for the exactness theorem.
+``theorem1`` holds the toy-model harness for the exactness theorem; ``interblock`` the joint
+mask, trigger and two-tree acceptance of inter-block speculation (Section 3.4).
 """
 from .binding import (  # noqa: F401
     build,
