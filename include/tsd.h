@@ -251,15 +251,69 @@ int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_
  *   topk_idx, topk_prob       device [batch, prev_branches, R, k]: stage 2 output of that pass.
  *   parent        device int32 [batch, max_nodes];  state device int32 [batch, max_nodes, R];
  *   node_prob     device fp32 [batch, max_nodes]: probability of the entry a node added (root 1);
- *   n_nodes       device int32 [batch].  Slots past n_nodes are copies of the root with parent 0.
+ *   n_nodes       device int32 [batch].  Slots past n_nodes are copies of the root hanging off it.
+ *   out_stride    branches per sequence in parent / state / node_prob (>= max_nodes): the tree
+ *                 may be a slice of a larger forest (pass pointers to its first branch);
+ *   node_base     added to every parent index written (the root still gets -1): the forest index
+ *                 of this tree's root;  0 and out_stride = max_nodes for a tree of its own;
+ *   enable        device uint8 [batch], nullable: 0 keeps that sequence's tree at its root
+ *                 (the inter-block trigger of Eq. 3).
  * R 1..128, k 1..8, width 1..32, depth >= 0, max_nodes 1..256.
  * ------------------------------------------------------------------------- */
 int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_t rows_per_branch, int32_t k,
                          const int32_t* prev_state, const int32_t* accepted_node,
                          const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
                          const int32_t* topk_idx, const float* topk_prob, int32_t width, int32_t depth,
-                         int32_t max_nodes, int32_t* parent, int32_t* state, float* node_prob,
-                         int32_t* n_nodes, uint32_t* status, tsd_stream_t stream);
+                         int32_t max_nodes, int32_t out_stride, int32_t node_base, const uint8_t* enable,
+                         int32_t* parent, int32_t* state, float* node_prob, int32_t* n_nodes,
+                         uint32_t* status, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Inter-block speculation (Section 3.4, Eq. 3, Appendix D): one pass verifies
+ * the tree of the current block B_t and a compact tree of the next block
+ * B_{t+1}.  Joint layout: branches [0, n_cur) = tree of B_t with its root at 0,
+ * branches [n_cur, n_branches) = tree of B_{t+1} with its root at n_cur; every
+ * branch is one block of R rows; parent[] holds forest indices and
+ * parent[n_cur] = -1.  None of the three calls below has a counterpart among the
+ * stages of the single-block path; they are its inter-block variant.
+ *
+ * tsd_build_interblock_vis writes the `vis` bitsets for tsd_build_branch_mask:
+ * the two roots read each other, a draft reads the other block's root, and
+ * nobody but the draft itself reads a draft (so a root's scores never depend on
+ * what was drafted).  n_cur = n_branches gives isolated branches.
+ *   vis  device uint64 [batch, n_branches, ceil(n_branches/64)].
+ *
+ * tsd_interblock_trigger evaluates Eq. 3 per sequence from the pass just
+ * verified: with c(b) = the largest confidence among the still-masked rows of
+ * node b, trigger = c(node_next) > c(node_cur[s]) or c(node_next) > tau; a next
+ * block without masked rows never triggers, a current block without masked
+ * rows always does.
+ *   state, conf  device [batch, n_branches, R] (int32 / fp32);
+ *   node_cur     device int32 [batch], nullable (= 0): the accepted node of B_t's tree;
+ *   node_next    index of B_{t+1}'s root;
+ *   trigger      device uint8 [batch];  top_conf device fp32 [batch, 2], nullable: c(cur), c(next).
+ *
+ * tsd_accept_joint_trees runs the acceptance of tsd_accept_trajectories on both
+ * trees in one launch.  Per-branch outputs (edge_valid, prefix_len) keep the
+ * forest layout [batch, n_branches]; per-tree outputs are tree-major:
+ * accepted_node, accepted_len, n_new_tokens [2, batch] and unmask_flag,
+ * unmask_tok [2, batch, R]; accepted_node is a forest index.  With
+ * n_cur = n_branches only tree 0 is written.  A parent outside its own tree sets
+ * TSD_STATUS_BAD_PARENT and invalidates that edge.
+ * ------------------------------------------------------------------------- */
+int tsd_build_interblock_vis(int32_t batch, int32_t n_branches, int32_t n_cur, uint64_t* vis,
+                             tsd_stream_t stream);
+int tsd_interblock_trigger(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+                           const int32_t* state, const float* conf, const int32_t* node_cur,
+                           int32_t node_next, int32_t mask_id, float tau, uint8_t* trigger,
+                           float* top_conf, uint32_t* status, tsd_stream_t stream);
+int tsd_accept_joint_trees(int32_t batch, int32_t n_branches, int32_t n_cur, int32_t rows_per_branch,
+                           const int32_t* parent, const int32_t* state, int32_t mask_id,
+                           const float* conf, const int32_t* top1_idx, int32_t top1_stride, float tau,
+                           int32_t rule, int32_t search, uint8_t* edge_valid, int32_t* prefix_len,
+                           int32_t* accepted_node, int32_t* accepted_len, int32_t* n_new_tokens,
+                           uint8_t* unmask_flag, int32_t* unmask_tok, uint32_t* status,
+                           tsd_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -27,6 +27,7 @@ EXPORTS = (
     "tsd_confidence_topk_workspace_bytes", "tsd_confidence_topk",
     "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
     "tsd_accept_trajectories", "tsd_build_draft_tree",
+    "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees",
 )
 
 
@@ -80,7 +81,12 @@ def lib():
         L.tsd_accept_trajectories.argtypes = [_i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
                                               _i32, _i32] + [_vp] * 9
         L.tsd_build_draft_tree.argtypes = [_i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32,
-                                           _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+                                           _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+        L.tsd_build_interblock_vis.argtypes = [_i32, _i32, _i32, _vp, _vp]
+        L.tsd_interblock_trigger.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp, _vp,
+                                             _vp]
+        L.tsd_accept_joint_trees.argtypes = [_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
+                                             _i32, _i32] + [_vp] * 9
         _lib = L
     return _lib
 
@@ -202,14 +208,58 @@ def tsd_accept_trajectories(parent, state, mask_id, conf, top1_idx, top1_stride,
     _check(rc, "tsd_accept_trajectories")
 
 
+def _slice_ptr(t, first):
+    """Address of branch `first` of sequence 0 in a contiguous [S, B, ...] tensor."""
+    return ctypes.c_void_p(t.data_ptr() + first * t.stride(1) * t.element_size())
+
+
 def tsd_build_draft_tree(prev_state, accepted_node, unmask_flag, unmask_tok, mask_id, topk_idx, topk_prob,
-                         width, depth, parent, state, node_prob, n_nodes, status=None, stream=None):
+                         width, depth, parent, state, node_prob, n_nodes, status=None, stream=None,
+                         first=0, max_nodes=None, enable=None):
     """prev_state [S,Bp,R]; topk_idx/topk_prob [S*Bp*R, k] (or any shape with that many entries);
-    outputs parent [S,B], state [S,B,R], node_prob [S,B], n_nodes [S]."""
+    outputs parent [S,B], state [S,B,R], node_prob [S,B], n_nodes [S].  With `first`/`max_nodes`
+    the tree fills branches [first, first + max_nodes) of the (larger) output arrays and its
+    parent indices count from `first`; `enable` uint8 [S] keeps a sequence's tree at its root."""
     S, Bp, R = prev_state.shape
     k = topk_idx.shape[-1]
+    B = state.shape[1]
+    max_nodes = B - first if max_nodes is None else int(max_nodes)
+    assert state.is_contiguous() and parent.is_contiguous() and node_prob.is_contiguous()
+    assert 0 <= first and first + max_nodes <= B
     rc = lib().tsd_build_draft_tree(
         S, Bp, R, k, _ptr(prev_state), _ptr(accepted_node), _ptr(unmask_flag), _ptr(unmask_tok), int(mask_id),
-        _ptr(topk_idx), _ptr(topk_prob), int(width), int(depth), int(state.shape[1]), _ptr(parent), _ptr(state),
-        _ptr(node_prob), _ptr(n_nodes), _ptr(status), _stream(stream))
+        _ptr(topk_idx), _ptr(topk_prob), int(width), int(depth), max_nodes, B, int(first), _ptr(enable),
+        _slice_ptr(parent, first), _slice_ptr(state, first), _slice_ptr(node_prob, first), _ptr(n_nodes),
+        _ptr(status), _stream(stream))
     _check(rc, "tsd_build_draft_tree")
+
+
+def tsd_build_interblock_vis(n_cur, vis, stream=None):
+    """vis uint64/int64 [S, B, ceil(B/64)] (written)."""
+    S, B, W = vis.shape
+    assert W == (B + 63) // 64 and vis.is_contiguous() and vis.element_size() == 8
+    _check(lib().tsd_build_interblock_vis(S, B, int(n_cur), _ptr(vis), _stream(stream)),
+           "tsd_build_interblock_vis")
+
+
+def tsd_interblock_trigger(state, conf, node_cur, node_next, mask_id, tau, trigger, top_conf=None,
+                           status=None, stream=None):
+    S, B, R = state.shape
+    rc = lib().tsd_interblock_trigger(S, B, R, _ptr(state), _ptr(conf), _ptr(node_cur), int(node_next),
+                                      int(mask_id), float(tau), _ptr(trigger), _ptr(top_conf), _ptr(status),
+                                      _stream(stream))
+    _check(rc, "tsd_interblock_trigger")
+
+
+def tsd_accept_joint_trees(parent, state, n_cur, mask_id, conf, top1_idx, top1_stride, tau, rule, search,
+                           edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens,
+                           unmask_flag, unmask_tok, status=None, stream=None):
+    """Forest layout: parent/edge_valid/prefix_len [S,B]; accepted_* and n_new_tokens [2,S];
+    unmask_* [2,S,R]."""
+    S, B, R = state.shape
+    rc = lib().tsd_accept_joint_trees(
+        S, B, int(n_cur), R, _ptr(parent), _ptr(state), int(mask_id), _ptr(conf), _ptr(top1_idx),
+        int(top1_stride), float(tau), int(rule), int(search), _ptr(edge_valid), _ptr(prefix_len),
+        _ptr(accepted_node), _ptr(accepted_len), _ptr(n_new_tokens), _ptr(unmask_flag), _ptr(unmask_tok),
+        _ptr(status), _stream(stream))
+    _check(rc, "tsd_accept_joint_trees")

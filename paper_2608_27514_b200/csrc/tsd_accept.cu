@@ -5,6 +5,10 @@
 // every node (what threshold decoding would unmask next), then the validity of every edge, both
 // as warp ballots over the block's rows; one thread then walks the tree (a few dozen nodes).
 // Integer and float compares only: the result is exact.
+//
+// The joint pass of inter-block speculation (Section 3.4) verifies two trees at once: branches
+// [0, n_cur) and [n_cur, B) of the same arrays.  blockIdx.y picks the tree; per-branch outputs
+// keep their position in the forest, per-tree outputs are tree-major ([2, batch, ...]).
 #include <limits.h>
 #include <math_constants.h>
 #include "tsd_common.cuh"
@@ -17,7 +21,7 @@ constexpr int kRowWords = kMaxRows / 32;
 constexpr int kAcceptThreads = 256;
 
 __global__ void __launch_bounds__(kAcceptThreads)
-accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
+accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
               int mask_id, const float* __restrict__ conf, const int32_t* __restrict__ top1,
               int top1_stride, float tau, int rule, int search, uint8_t* __restrict__ edge_valid,
               int32_t* __restrict__ prefix_len, int32_t* __restrict__ accepted_node,
@@ -28,12 +32,16 @@ accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
   __shared__ uint8_t s_valid[kMaxBranches];
   __shared__ int s_par[kMaxBranches];
   __shared__ int s_acc;
-  const int s = blockIdx.x;
+  const int s = blockIdx.x, tree = blockIdx.y, batch = gridDim.x;
+  const int lo = tree ? n_cur : 0;          // first branch of this tree = its root
+  const int B = tree ? B_all - n_cur : n_cur;  // its size (0: nothing to verify)
+  const size_t ts = (size_t)tree * batch + s;  // slot in the tree-major outputs
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   const unsigned full = 0xffffffffu;
-  const int32_t* st = state + (size_t)s * B * R;
-  const float* cf = conf + (size_t)s * B * R;
-  const int32_t* t1 = top1 + (size_t)s * B * R * top1_stride;
+  if (B <= 0) return;
+  const int32_t* st = state + ((size_t)s * B_all + lo) * R;
+  const float* cf = conf + ((size_t)s * B_all + lo) * R;
+  const int32_t* t1 = top1 + ((size_t)s * B_all + lo) * R * top1_stride;
   const int words = (R + 31) / 32;
 
   // decode rule U(p) for every node
@@ -73,7 +81,11 @@ accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
     if (lane == 0) {
 #pragma unroll
       for (int w = 0; w < kRowWords; ++w) s_u[p][w] = hi[w];
-      int par = p == 0 ? -1 : parent[(size_t)s * B + p];
+      int par = -1;
+      if (p > 0) {
+        const int raw = parent[(size_t)s * B_all + lo + p];  // forest index
+        par = raw >= lo ? raw - lo : -1;                      // local to the tree
+      }
       if (p > 0 && (par < 0 || par >= p)) {
         if (status) atomicOr(status, TSD_STATUS_BAD_PARENT);
         par = -1;  // treated as an invalid edge hanging off nothing
@@ -116,8 +128,8 @@ accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
   if (threadIdx.x == 0) {
     // prefix_len is read back from the global array this block has just written; a node's depth
     // is found by walking its parents (trees are a few levels deep)
-    int32_t* pl = prefix_len + (size_t)s * B;
-    uint8_t* ev = edge_valid + (size_t)s * B;
+    int32_t* pl = prefix_len + (size_t)s * B_all + lo;
+    uint8_t* ev = edge_valid + (size_t)s * B_all + lo;
     int acc = 0, acc_depth = 0;
     pl[0] = 0;
     ev[0] = 1;
@@ -141,8 +153,8 @@ accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
         ++acc_depth;
       }
     }
-    accepted_node[s] = acc;
-    accepted_len[s] = acc_depth;
+    accepted_node[ts] = lo + acc;  // index in the forest
+    accepted_len[ts] = acc_depth;
     s_acc = acc;
   }
   __syncthreads();
@@ -158,25 +170,23 @@ accept_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
       gained += __popc(__ballot_sync(full, fa)) - __popc(__ballot_sync(full, f0));
       if (r < R) {
         const bool in_u = (s_u[acc][w] >> lane) & 1u;
-        unmask_flag[(size_t)s * R + r] = in_u ? 1 : 0;
-        unmask_tok[(size_t)s * R + r] = in_u ? t1[(size_t)(acc * R + r) * top1_stride] : -1;
+        unmask_flag[ts * R + r] = in_u ? 1 : 0;
+        unmask_tok[ts * R + r] = in_u ? t1[(size_t)(acc * R + r) * top1_stride] : -1;
       }
     }
-    if (lane == 0) n_new_tokens[s] = gained;
+    if (lane == 0) n_new_tokens[ts] = gained;
   }
 }
 
 }  // namespace tsd
 
-extern "C" int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
-                                       const int32_t* parent, const int32_t* state, int32_t mask_id,
-                                       const float* conf, const int32_t* top1_idx, int32_t top1_stride,
-                                       float tau, int32_t rule, int32_t search, uint8_t* edge_valid,
-                                       int32_t* prefix_len, int32_t* accepted_node,
-                                       int32_t* accepted_len, int32_t* n_new_tokens,
-                                       uint8_t* unmask_flag, int32_t* unmask_tok, uint32_t* status,
-                                       tsd_stream_t stream) {
-  if (batch < 0 || n_branches < 1 || n_branches > tsd::kMaxBranches || rows_per_branch < 1 ||
+static int accept_launch(int32_t batch, int32_t n_branches, int32_t n_cur, int32_t rows_per_branch,
+                         const int32_t* parent, const int32_t* state, int32_t mask_id, const float* conf,
+                         const int32_t* top1_idx, int32_t top1_stride, float tau, int32_t rule,
+                         int32_t search, uint8_t* edge_valid, int32_t* prefix_len, int32_t* accepted_node,
+                         int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
+                         int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream) {
+  if (batch < 0 || n_cur < 1 || n_cur > n_branches || n_branches < 1 || n_branches > tsd::kMaxBranches || rows_per_branch < 1 ||
       rows_per_branch > tsd::kMaxRows || top1_stride < 1)
     return TSD_ERR_INVALID_ARG;
   if (rule != TSD_ACCEPT_EXACT && rule != TSD_ACCEPT_TOP1) return TSD_ERR_INVALID_ARG;
@@ -186,11 +196,37 @@ extern "C" int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_
   if (!parent || !state || !conf || !top1_idx || !edge_valid || !prefix_len || !accepted_node ||
       !accepted_len || !n_new_tokens || !unmask_flag || !unmask_tok)
     return TSD_ERR_INVALID_ARG;
-  tsd::accept_kernel<<<batch, tsd::kAcceptThreads, 0, stream>>>(
-      n_branches, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
+  const dim3 grid(batch, n_cur < n_branches ? 2 : 1);
+  tsd::accept_kernel<<<grid, tsd::kAcceptThreads, 0, stream>>>(
+      n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
       search, edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
       unmask_tok, status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return tsd::cuda_fail(e, "accept_kernel");
   return TSD_OK;
+}
+
+extern "C" int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+                                       const int32_t* parent, const int32_t* state, int32_t mask_id,
+                                       const float* conf, const int32_t* top1_idx, int32_t top1_stride,
+                                       float tau, int32_t rule, int32_t search, uint8_t* edge_valid,
+                                       int32_t* prefix_len, int32_t* accepted_node,
+                                       int32_t* accepted_len, int32_t* n_new_tokens,
+                                       uint8_t* unmask_flag, int32_t* unmask_tok, uint32_t* status,
+                                       tsd_stream_t stream) {
+  return accept_launch(batch, n_branches, n_branches, rows_per_branch, parent, state, mask_id, conf, top1_idx,
+                       top1_stride, tau, rule, search, edge_valid, prefix_len, accepted_node, accepted_len,
+                       n_new_tokens, unmask_flag, unmask_tok, status, stream);
+}
+
+extern "C" int tsd_accept_joint_trees(int32_t batch, int32_t n_branches, int32_t n_cur,
+                                      int32_t rows_per_branch, const int32_t* parent, const int32_t* state,
+                                      int32_t mask_id, const float* conf, const int32_t* top1_idx,
+                                      int32_t top1_stride, float tau, int32_t rule, int32_t search,
+                                      uint8_t* edge_valid, int32_t* prefix_len, int32_t* accepted_node,
+                                      int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
+                                      int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream) {
+  return accept_launch(batch, n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx,
+                       top1_stride, tau, rule, search, edge_valid, prefix_len, accepted_node, accepted_len,
+                       n_new_tokens, unmask_flag, unmask_tok, status, stream);
 }

@@ -12,8 +12,13 @@
 //              frontier; the tree stops at max_nodes nodes.
 // Ties go to the lower row, then the lower rank, then the earlier child.  Lanes own rows
 // (row = lane + 32 i); every selection is a warp arg-best reduction, so the result is exact and
-// deterministic.  Unused node slots are copies of the root hanging off node 0 (an empty delta is
+// deterministic.  Unused node slots are copies of the root hanging off the root (an empty delta is
 // never accepted).
+//
+// For the joint pass of inter-block speculation (Section 3.4) the tree can be written into a slice
+// of a larger forest: `out_stride` branches per sequence in the output arrays, `node_base` added
+// to every parent index, and a per-sequence `enable` byte (the trigger of Eq. 3) that, when 0,
+// leaves the tree at its root.
 #include <limits.h>
 #include <math_constants.h>
 #include "tsd_common.cuh"
@@ -53,7 +58,8 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
                         const int32_t* __restrict__ accepted_node, const uint8_t* __restrict__ unmask_flag,
                         const int32_t* __restrict__ unmask_tok, int mask_id,
                         const int32_t* __restrict__ topk_idx, const float* __restrict__ topk_prob, int W,
-                        int D, int max_nodes, int32_t* __restrict__ parent, int32_t* __restrict__ state,
+                        int D, int max_nodes, int out_stride, int node_base,
+                        const uint8_t* __restrict__ enable, int32_t* __restrict__ parent, int32_t* __restrict__ state,
                         float* __restrict__ node_prob, int32_t* __restrict__ n_nodes,
                         uint32_t* __restrict__ status) {
   __shared__ int s_front[kTreeMaxWidth];
@@ -69,9 +75,10 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
   const size_t src = ((size_t)s * prev_branches + acc) * R;  // rows of the accepted node
   const int32_t* idx = topk_idx + src * k;
   const float* prb = topk_prob + src * k;
-  int32_t* st = state + (size_t)s * max_nodes * R;
-  int32_t* par = parent + (size_t)s * max_nodes;
-  float* np_ = node_prob + (size_t)s * max_nodes;
+  int32_t* st = state + (size_t)s * out_stride * R;
+  int32_t* par = parent + (size_t)s * out_stride;
+  float* np_ = node_prob + (size_t)s * out_stride;
+  if (enable && !enable[s]) D = 0;
 
   // next root = accepted state + its unmask set; every node slot starts as a copy of it
   bool root_masked[kTreeRowsPerLane];
@@ -87,7 +94,7 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
     }
   }
   for (int b = lane; b < max_nodes; b += 32) {
-    par[b] = b == 0 ? -1 : 0;
+    par[b] = b == 0 ? -1 : node_base;
     np_[b] = b == 0 ? 1.f : 0.f;
   }
   // the pool lives in registers (this lane's rows x k) and the nodes' masked-row sets in shared
@@ -172,7 +179,7 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
     __syncwarp();
     if (pos < keep) {
       s_front[pos] = n + pos;
-      par[n + pos] = my_par;
+      par[n + pos] = node_base + my_par;
       np_[n + pos] = my_p;
     }
     // materialise the kept children: node = copy of its parent + one filled row
@@ -203,12 +210,13 @@ extern "C" int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_
                                     const int32_t* prev_state, const int32_t* accepted_node,
                                     const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
                                     const int32_t* topk_idx, const float* topk_prob, int32_t width,
-                                    int32_t depth, int32_t max_nodes, int32_t* parent, int32_t* state,
-                                    float* node_prob, int32_t* n_nodes, uint32_t* status,
+                                    int32_t depth, int32_t max_nodes, int32_t out_stride,
+                                    int32_t node_base, const uint8_t* enable, int32_t* parent,
+                                    int32_t* state, float* node_prob, int32_t* n_nodes, uint32_t* status,
                                     tsd_stream_t stream) {
   if (batch < 0 || prev_branches < 1 || rows_per_branch < 1 || rows_per_branch > tsd::kTreeMaxRows || k < 1 ||
       k > tsd::kTreeMaxK || width < 1 || width > tsd::kTreeMaxWidth || depth < 0 || max_nodes < 1 ||
-      max_nodes > 256)
+      max_nodes > 256 || out_stride < max_nodes || node_base < 0)
     return TSD_ERR_INVALID_ARG;
   if ((unmask_flag == nullptr) != (unmask_tok == nullptr)) return TSD_ERR_INVALID_ARG;
   if (batch == 0) return TSD_OK;
@@ -216,7 +224,8 @@ extern "C" int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_
     return TSD_ERR_INVALID_ARG;
   tsd::build_draft_tree_kernel<<<batch, 32, 0, stream>>>(
       prev_branches, rows_per_branch, k, prev_state, accepted_node, unmask_flag, unmask_tok, mask_id, topk_idx,
-      topk_prob, width, depth, max_nodes, parent, state, node_prob, n_nodes, status);
+      topk_prob, width, depth, max_nodes, out_stride, node_base, enable, parent, state, node_prob, n_nodes,
+      status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return tsd::cuda_fail(e, "build_draft_tree_kernel");
   return TSD_OK;

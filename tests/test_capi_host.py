@@ -121,8 +121,9 @@ def test_tree_validation(lib):
     p = ctypes.c_void_p(4096)
     f = lib.tsd_build_draft_tree
 
-    def call(S=1, Bp=4, R=32, k=3, prev=p, flag=p, tok=p, W=2, D=2, B_=4):
-        return f(S, Bp, R, k, prev, p, flag, tok, 99, p, p, W, D, B_, p, p, p, p, None, None)
+    def call(S=1, Bp=4, R=32, k=3, prev=p, flag=p, tok=p, W=2, D=2, B_=4, stride=None, base=0):
+        return f(S, Bp, R, k, prev, p, flag, tok, 99, p, p, W, D, B_, B_ if stride is None else stride, base,
+                 None, p, p, p, p, None, None)
     assert call(R=129) == B.TSD_ERR_INVALID_ARG
     assert call(k=9) == B.TSD_ERR_INVALID_ARG
     assert call(W=0) == B.TSD_ERR_INVALID_ARG
@@ -130,4 +131,28 @@ def test_tree_validation(lib):
     assert call(B_=257) == B.TSD_ERR_INVALID_ARG
     assert call(flag=None) == B.TSD_ERR_INVALID_ARG      # flag without tokens
     assert call(prev=None) == B.TSD_ERR_INVALID_ARG
+    assert call(stride=3) == B.TSD_ERR_INVALID_ARG       # forest narrower than the tree
+    assert call(base=-1) == B.TSD_ERR_INVALID_ARG
     assert call(S=0) == B.TSD_OK
+
+
+def test_interblock_validation(lib):
+    p = ctypes.c_void_p(4096)
+    assert lib.tsd_build_interblock_vis(1, 8, 0, p, None) == B.TSD_ERR_INVALID_ARG    # no current tree
+    assert lib.tsd_build_interblock_vis(1, 8, 9, p, None) == B.TSD_ERR_INVALID_ARG
+    assert lib.tsd_build_interblock_vis(1, 257, 4, p, None) == B.TSD_ERR_INVALID_ARG
+    assert lib.tsd_build_interblock_vis(1, 8, 4, None, None) == B.TSD_ERR_INVALID_ARG
+    assert lib.tsd_build_interblock_vis(0, 8, 4, None, None) == B.TSD_OK
+    trig = lib.tsd_interblock_trigger
+    assert trig(1, 8, 32, p, p, None, 8, 99, 0.9, p, None, None, None) == B.TSD_ERR_INVALID_ARG  # root outside
+    assert trig(1, 8, 32, p, p, None, 4, 99, float("nan"), p, None, None, None) == B.TSD_ERR_INVALID_ARG
+    assert trig(1, 8, 32, None, p, None, 4, 99, 0.9, p, None, None, None) == B.TSD_ERR_INVALID_ARG
+    assert trig(0, 8, 32, None, None, None, 4, 99, 0.9, None, None, None, None) == B.TSD_OK
+    acc = lib.tsd_accept_joint_trees
+
+    def call(B_=8, n_cur=4, R=32, rule=0):
+        return acc(1, B_, n_cur, R, p, p, 99, p, p, 1, 0.9, rule, 0, *([p] * 7), None, None)
+    assert call(n_cur=0) == B.TSD_ERR_INVALID_ARG
+    assert call(n_cur=9) == B.TSD_ERR_INVALID_ARG
+    assert call(R=129) == B.TSD_ERR_INVALID_ARG
+    assert call(rule=2) == B.TSD_ERR_INVALID_ARG
