@@ -16,5 +16,6 @@ from .binding import (  # noqa: F401
     confidence_topk,
     decode_rule,
     accept,
+    draft_token_prob,
     build_draft_tree,
 )

@@ -109,16 +109,21 @@ def decode_rule(state, mask_id, conf, top1, tau):
     return flag, tok
 
 
-def accept(parent, state, mask_id, conf, top1, tau, rule=0, search=0):
-    """parent [S,B], state [S,B,R], conf [S,B,R] fp32, top1 [S,B,R] ->
-    dict of edge_valid, prefix_len, accepted_node, accepted_len,
-    n_new_tokens, unmask_flag, unmask_tok."""
+def accept(parent, state, mask_id, conf, top1, tau, rule=0, search=0, topk_m=1, draft_prob=None):
+    """parent [S,B], state [S,B,R], conf [S,B,R] fp32, top1 [S,B,R] or the
+    candidate lists [S,B,R,k] (entry 0 = arg-max; rule 2 tests the first
+    topk_m), draft_prob fp32 [S,B,R] (rule 3) -> dict of edge_valid,
+    prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
+    unmask_tok."""
     parent = _arr(parent, np.int32)
     state = _arr(state, np.int32)
     conf = _arr(conf, np.float32)
     top1 = _arr(top1, np.int32)
+    draft_prob = _arr(draft_prob, np.float32)
     S, B, R = state.shape
-    assert parent.shape == (S, B) and conf.shape == (S, B, R) and top1.shape == (S, B, R)
+    stride = 1 if top1.ndim == 3 else top1.shape[3]
+    assert parent.shape == (S, B) and conf.shape == (S, B, R) and top1.shape[:3] == (S, B, R)
+    assert 1 <= topk_m <= stride and (rule != 3 or draft_prob.shape == (S, B, R))
     o = dict(
         edge_valid=np.empty((S, B), np.uint8),
         prefix_len=np.empty((S, B), np.int32),
@@ -130,11 +135,26 @@ def accept(parent, state, mask_id, conf, top1, tau, rule=0, search=0):
     )
     _load().oracle_accept(
         S, B, R, _ptr(parent), _ptr(state), ctypes.c_int32(mask_id), _ptr(conf),
-        _ptr(top1), ctypes.c_int64(1), ctypes.c_float(tau), int(rule), int(search),
+        _ptr(top1), ctypes.c_int64(stride), int(topk_m), _ptr(draft_prob), ctypes.c_float(tau),
+        int(rule), int(search),
         _ptr(o["edge_valid"]), _ptr(o["prefix_len"]), _ptr(o["accepted_node"]),
         _ptr(o["accepted_len"]), _ptr(o["n_new_tokens"]), _ptr(o["unmask_flag"]),
         _ptr(o["unmask_tok"]))
     return o
+
+
+def draft_token_prob(logits, parent, state, mask_id):
+    """logits [S,B,R,V], parent [S,B], state [S,B,R] -> fp64 [S,B,R]: probability of each drafted
+    token under its parent's distribution at that row (0 where the child adds nothing)."""
+    logits = _arr(logits, np.float32)
+    parent = _arr(parent, np.int32)
+    state = _arr(state, np.int32)
+    S, B, R, V = logits.shape
+    assert parent.shape == (S, B) and state.shape == (S, B, R)
+    out = np.empty((S, B, R), dtype=np.float64)
+    _load().oracle_draft_token_prob(S, B, R, V, _ptr(logits), _ptr(parent), _ptr(state),
+                                    ctypes.c_int32(mask_id), _ptr(out))
+    return out
 
 
 def build_draft_tree(root_state, mask_id, topk_idx, topk_prob, W, D, max_nodes):

@@ -16,7 +16,9 @@
  *   oracle_confidence_topk   Eq. 2 (confidence) and the top-k candidates of Section 3.2
  *   oracle_decode_rule       Alg. 1 Phase 1 (H = {conf > tau}) with the top-1
  *                            fallback of Eqs. 6-7
- *   oracle_accept            Section 3.3 "Verification procedure" (greedy / longest path)
+ *   oracle_accept            Section 3.3 "Verification procedure" (greedy / longest path;
+ *                            exact, top-1, top-k-membership and probability tests)
+ *   oracle_draft_token_prob  probability of a drafted token under its parent (Eq. 2's softmax)
  *   oracle_build_draft_tree  Alg. 1 Phase 2 (the step before the path; built after it)
  *
  * Pins (tests/test_oracle_*.py): textbook attention for one branch, plain
@@ -230,6 +232,17 @@ int oracle_decode_rule(int R, const int32_t* state, int32_t mask_id,
  * had already filled or re-masks one; a malformed or empty delta is invalid.
  *   rule 0 (EXACT): D(c) == U(parent) as sets of (row, token)
  *   rule 1 (TOP1) : every (r, t) in D(c) has t == top1[parent][r]
+ *   rule 2 (TOPK) : every (r, t) in D(c) has t among the parent's topk_m most
+ *                   probable tokens at r ("fall within top-k")
+ *   rule 3 (PROB) : every (r, t) in D(c) has draft_prob[c][r] > tau, where
+ *                   draft_prob[c][r] is the probability the parent's
+ *                   distribution at r gives to t ("exceed tau"; strict, as
+ *                   in Alg. 1)
+ * Rules 1-3 admit trajectory drift (Section 4, last paragraph); only rule 0
+ * is the test of Theorem 1.  top1 holds, per (node, row), the candidate
+ * tokens in descending probability, top1_stride apart; entry 0 is the arg-max.
+ * An edge whose parent index lies outside [0, c) is not an edge of the tree:
+ * it is invalid and c counts as a depth-1 node with no valid prefix.
  * prefix_len[b] = number of leading valid edges on the path root -> b.
  * search 0 (GREEDY): from the root, move to the lowest-index valid child
  *                    until there is none.
@@ -240,7 +253,8 @@ int oracle_decode_rule(int R, const int32_t* state, int32_t mask_id,
  * ---------------------------------------------------------------------- */
 void oracle_accept(int S, int B, int R, const int32_t* parent,
                    const int32_t* state, int32_t mask_id, const float* conf,
-                   const int32_t* top1, int64_t top1_stride, float tau,
+                   const int32_t* top1, int64_t top1_stride, int topk_m,
+                   const float* draft_prob, float tau,
                    int rule, int search, uint8_t* edge_valid,
                    int32_t* prefix_len, int32_t* accepted_node,
                    int32_t* accepted_len, int32_t* n_new_tokens,
@@ -258,6 +272,12 @@ void oracle_accept(int S, int B, int R, const int32_t* parent,
     depth[0] = 0;
     for (int c = 1; c < B; ++c) {
       const int p = par[c];
+      if (p < 0 || p >= c) {
+        ev[c] = 0;
+        depth[c] = 1;
+        pl[c] = 0;
+        continue;
+      }
       const int32_t* sp = state + ((int64_t)s * B + p) * R;
       const int32_t* sc = state + ((int64_t)s * B + c) * R;
       const float* cp = conf + ((int64_t)s * B + p) * R;
@@ -279,8 +299,15 @@ void oracle_accept(int S, int B, int R, const int32_t* parent,
         ++n_delta;
         if (rule == 0) {
           if (!uflag[r] || utok[r] != sc[r]) ok = 0;
-        } else {
+        } else if (rule == 1) {
           if (t1[r] != sc[r]) ok = 0;
+        } else if (rule == 2) {
+          const int32_t* cand = top1 + (((int64_t)s * B + p) * R + r) * top1_stride;
+          int found = 0;
+          for (int j = 0; j < topk_m; ++j) found |= (cand[j] == sc[r]);
+          if (!found) ok = 0;
+        } else {
+          if (!(draft_prob[((int64_t)s * B + c) * R + r] > tau)) ok = 0;
         }
       }
       ev[c] = (uint8_t)(ok && !malformed && n_delta > 0);
@@ -323,6 +350,38 @@ void oracle_accept(int S, int B, int R, const int32_t* parent,
   free(utok);
   free(t1);
   free(depth);
+}
+
+/* ------------------------------------------------------------------------
+ * Probability of every drafted token under its parent's distribution
+ * (the quantity the "exceed tau" reading of Section 3.3 tests): for child c,
+ * row r in D(c) with token t,
+ *   out[c][r] = exp(z_t - max z) / sum_v exp(z_v - max z),  z = logits[parent(c)][r]
+ * (Eq. 2's softmax).  Rows outside D(c), the root, nodes with a parent index
+ * outside [0, c) and tokens outside [0, V) get 0.
+ * logits [S,B,R,V] fp32, out [S,B,R] fp64.
+ * ---------------------------------------------------------------------- */
+void oracle_draft_token_prob(int S, int B, int R, int V, const float* logits,
+                             const int32_t* parent, const int32_t* state,
+                             int32_t mask_id, double* out) {
+  for (int s = 0; s < S; ++s)
+    for (int c = 0; c < B; ++c) {
+      const int p = parent[(int64_t)s * B + c];
+      for (int r = 0; r < R; ++r) {
+        double* o = out + ((int64_t)s * B + c) * R + r;
+        *o = 0.0;
+        if (c == 0 || p < 0 || p >= c) continue;
+        const int32_t tp = state[((int64_t)s * B + p) * R + r];
+        const int32_t tc = state[((int64_t)s * B + c) * R + r];
+        if (tp != mask_id || tc == mask_id || tc < 0 || tc >= V) continue;
+        const float* z = logits + (((int64_t)s * B + p) * R + r) * (int64_t)V;
+        double zmax = -INFINITY, sum = 0.0;
+        for (int v = 0; v < V; ++v)
+          if ((double)z[v] > zmax) zmax = (double)z[v];
+        for (int v = 0; v < V; ++v) sum += exp((double)z[v] - zmax);
+        *o = exp((double)z[tc] - zmax) / sum;
+      }
+    }
 }
 
 /* ------------------------------------------------------------------------

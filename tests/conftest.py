@@ -30,9 +30,12 @@ def load_accept_cases():
             top1=np.array(c["top1"], dtype=np.int32)[None],
             tau=float(c["tau"]),
             mask_id=99,
+            topk=None if "topk" not in c else np.array(c["topk"], dtype=np.int32)[None],
+            topk_m=int(c.get("topk_m", 1)),
+            draft_prob=None if "draft_prob" not in c else np.array(c["draft_prob"], dtype=np.float32)[None],
         )
         for run in c["runs"]:
-            out.append(dict(base, rule={"EXACT": 0, "TOP1": 1}[run["rule"]],
+            out.append(dict(base, rule={"EXACT": 0, "TOP1": 1, "TOPK": 2, "PROB": 3}[run["rule"]],
                             search={"GREEDY": 0, "LONGEST": 1}[run["search"]],
                             expect=run, id="%s-%s-%s" % (c["name"], run["rule"], run["search"])))
     return out
