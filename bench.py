@@ -334,6 +334,13 @@ def main():
         step, attn, vi = sets[i % n_copies]
         step.accept(vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
 
+    def f_acc_prob(i):
+        # the relaxed reading of the test (probability of the drafted token above tau, longest path),
+        # with its gather from the logits; timed for context, the step uses the exact test
+        step, attn, vi = sets[i % n_copies]
+        step.accept_relaxed(vi["parent"], vi["state"], vi["mask_id"], cfg.tau, B.TSD_ACCEPT_PROB,
+                            B.TSD_SEARCH_LONGEST, vi["logits"])
+
     # the step before the path (Alg. 1 tree construction fused with the root update), timed for
     # context only: it is not part of the step
     tree_out = dict(parent=torch.empty((cfg.S, cfg.B), dtype=torch.int32, device=dev),
@@ -367,6 +374,7 @@ def main():
     # the tensor-heavy stage last: it drives the GPU into its power cap, which would lower the
     # clocks the other two are measured at
     t_tree = time_stage(f_tree, 0.05)
+    t_acc_prob = time_stage(f_acc_prob, 0.05)
     t_acc, t_topk, t_attn = time_stage(f_acc, 0.05), time_stage(f_topk), time_stage(f_attn)
     if ib is not None:
         ib["seconds"] = time_stage(f_ib)
@@ -424,6 +432,8 @@ def main():
         topk=dict(seconds=t_topk, bound="hbm", roofline_seconds=alg["topk_bytes"] / (pk["hbm_gbs"] * 1e9),
                   frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9),
         accept=dict(seconds=t_acc),
+        accept_relaxed_prob_longest=dict(seconds=t_acc_prob, note="Section 3.3's 'exceed tau' reading with the "
+                                         "gather of the drafted tokens' probabilities; not part of the step"),
         tree_build_next_step=dict(seconds=t_tree, note="Alg. 1 tree construction (W3 D3) for the next step; not part of the step"),
     )
     if ib is not None:

@@ -54,7 +54,16 @@ typedef enum { TSD_F32 = 0, TSD_BF16 = 1 } tsd_dtype;
  * its parent; this is the test under which Theorem 1 holds.  TOP1: every token
  * the child adds is its parent's top prediction at that row (the literal
  * "tokens match the model's top predictions"; admits trajectory drift). */
-typedef enum { TSD_ACCEPT_EXACT = 0, TSD_ACCEPT_TOP1 = 1 } tsd_accept_rule;
+typedef enum {
+  TSD_ACCEPT_EXACT = 0,
+  TSD_ACCEPT_TOP1 = 1,
+  /* The two relaxed readings of the same sentence ("or fall within top-k / exceed tau"), served
+   * by tsd_accept_relaxed only.  TOPK: every token the child adds is among its parent's first
+   * topk_m candidates at that row.  PROB: every token the child adds has probability > tau
+   * (strictly) under its parent's distribution at that row.  Both admit drift. */
+  TSD_ACCEPT_TOPK = 2,
+  TSD_ACCEPT_PROB = 3
+} tsd_accept_rule;
 
 /* Greedy search takes the first valid continuation per level; longest-path
  * search takes the deepest fully valid path (Section 3.3). */
@@ -293,7 +302,8 @@ int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_t rows_per_
  *   node_next    index of B_{t+1}'s root;
  *   trigger      device uint8 [batch];  top_conf device fp32 [batch, 2], nullable: c(cur), c(next).
  *
- * tsd_accept_joint_trees runs the acceptance of tsd_accept_trajectories on both
+ * tsd_accept_joint_trees runs the acceptance of tsd_accept_trajectories (rules
+ * EXACT and TOP1) on both
  * trees in one launch.  Per-branch outputs (edge_valid, prefix_len) keep the
  * forest layout [batch, n_branches]; per-tree outputs are tree-major:
  * accepted_node, accepted_len, n_new_tokens [2, batch] and unmask_flag,
@@ -303,6 +313,35 @@ int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_t rows_per_
  * ------------------------------------------------------------------------- */
 int tsd_build_interblock_vis(int32_t batch, int32_t n_branches, int32_t n_cur, uint64_t* vis,
                              tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Acceptance under any of the four rules (Section 3.3, "Verification
+ * procedure": tokens "match the model's top predictions (or fall within top-k /
+ * exceed tau)"), for one tree (n_cur = n_branches) or the two trees of a joint
+ * pass; outputs laid out as for tsd_accept_joint_trees.  Combined with
+ * TSD_SEARCH_LONGEST this is the longest-path search under trajectory drift.
+ *
+ *   topk_idx     device int32, candidates per (node, row) in descending probability,
+ *                topk_stride apart (stage 2's topk_idx); entry 0 is the top prediction;
+ *   topk_m       1..topk_stride: how many of them count for TSD_ACCEPT_TOPK;
+ *   logits       device, nullable unless rule = TSD_ACCEPT_PROB: the logits of the pass,
+ *                [batch * n_branches * R, vocab], rows row_stride elements apart, dtype as given;
+ *   lse          device fp32 [batch * n_branches * R]: stage 2's log-sum-exp of each row
+ *                (required with logits);
+ *   draft_prob   device fp32 [batch, n_branches, R], nullable: probability, under the parent's
+ *                distribution, of the token each node adds at each row, exp(logit - lse) in
+ *                fp32 (0 where the node adds nothing); written whenever logits are given.  The
+ *                PROB rule compares exactly these fp32 values with tau.
+ * A drafted token outside [0, vocab) has probability 0.
+ * ------------------------------------------------------------------------- */
+int tsd_accept_relaxed(int32_t batch, int32_t n_branches, int32_t n_cur, int32_t rows_per_branch,
+                       const int32_t* parent, const int32_t* state, int32_t mask_id, const float* conf,
+                       const int32_t* topk_idx, int32_t topk_stride, int32_t topk_m, const void* logits,
+                       int32_t dtype, int64_t vocab, int64_t row_stride, const float* lse, float tau,
+                       int32_t rule, int32_t search, uint8_t* edge_valid, int32_t* prefix_len,
+                       int32_t* accepted_node, int32_t* accepted_len, int32_t* n_new_tokens,
+                       uint8_t* unmask_flag, int32_t* unmask_tok, float* draft_prob, uint32_t* status,
+                       tsd_stream_t stream);
 int tsd_interblock_trigger(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
                            const int32_t* state, const float* conf, const int32_t* node_cur,
                            int32_t node_next, int32_t mask_id, float tau, uint8_t* trigger,

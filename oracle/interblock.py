@@ -56,7 +56,7 @@ def interblock_trigger(state_cur, conf_cur, state_next, conf_next, mask_id, tau)
     return bool(c_next > c_cur or c_next > np.float32(tau))
 
 
-def joint_accept(parent, state, n_cur, mask_id, conf, top1, tau, rule=0, search=0):
+def joint_accept(parent, state, n_cur, mask_id, conf, top1, tau, rule=0, search=0, topk_m=1, draft_prob=None):
     """Acceptance of the two trees of a joint pass, each by the single-tree procedure of
     Section 3.3 on its own branches.  parent [S,B] holds forest indices (parent[:, n_cur] = -1).
     Returns per-branch arrays over the forest and per-tree arrays with a leading axis of 2
@@ -76,7 +76,8 @@ def joint_accept(parent, state, n_cur, mask_id, conf, top1, tau, rule=0, search=
         par = parent[:, lo:hi].copy()
         par[:, 1:] -= lo                 # indices local to the tree
         par[:, 0] = -1
-        o = binding.accept(par, state[:, lo:hi], mask_id, conf[:, lo:hi], top1[:, lo:hi], tau, rule, search)
+        o = binding.accept(par, state[:, lo:hi], mask_id, conf[:, lo:hi], top1[:, lo:hi], tau, rule, search,
+                           topk_m, None if draft_prob is None else np.asarray(draft_prob)[:, lo:hi])
         out["edge_valid"][:, lo:hi] = o["edge_valid"]
         out["prefix_len"][:, lo:hi] = o["prefix_len"]
         out["accepted_node"][t] = o["accepted_node"] + lo

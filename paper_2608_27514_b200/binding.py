@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtsd.so")
 
 TSD_F32, TSD_BF16 = 0, 1
-TSD_ACCEPT_EXACT, TSD_ACCEPT_TOP1 = 0, 1
+TSD_ACCEPT_EXACT, TSD_ACCEPT_TOP1, TSD_ACCEPT_TOPK, TSD_ACCEPT_PROB = 0, 1, 2, 3
 TSD_SEARCH_GREEDY, TSD_SEARCH_LONGEST = 0, 1
 TSD_ATTN_FORCE_SIMT = 0x1
 TSD_OK, TSD_ERR_INVALID_ARG, TSD_ERR_UNSUPPORTED, TSD_ERR_WORKSPACE = 0, -1, -2, -3
@@ -27,7 +27,7 @@ EXPORTS = (
     "tsd_confidence_topk_workspace_bytes", "tsd_confidence_topk",
     "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
     "tsd_accept_trajectories", "tsd_build_draft_tree",
-    "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees",
+    "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees", "tsd_accept_relaxed",
 )
 
 
@@ -87,6 +87,8 @@ def lib():
                                              _vp]
         L.tsd_accept_joint_trees.argtypes = [_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _f32,
                                              _i32, _i32] + [_vp] * 9
+        L.tsd_accept_relaxed.argtypes = ([_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _vp, _i32,
+                                          _i64, _i64, _vp, _f32, _i32, _i32] + [_vp] * 10)
         _lib = L
     return _lib
 
@@ -263,3 +265,21 @@ def tsd_accept_joint_trees(parent, state, n_cur, mask_id, conf, top1_idx, top1_s
         _ptr(accepted_node), _ptr(accepted_len), _ptr(n_new_tokens), _ptr(unmask_flag), _ptr(unmask_tok),
         _ptr(status), _stream(stream))
     _check(rc, "tsd_accept_joint_trees")
+
+
+def tsd_accept_relaxed(parent, state, n_cur, mask_id, conf, topk_idx, topk_m, logits, lse, tau, rule, search,
+                       edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
+                       unmask_tok, draft_prob=None, status=None, stream=None):
+    """Any of the four rules on one tree (n_cur = B) or two; topk_idx [S,B,R,k]; logits
+    [S*B*R, V] (or None) with lse [S*B*R]; per-tree outputs [2,S,...] (row 0 only for one tree)."""
+    S, B, R = state.shape
+    if logits is not None:
+        assert logits.dim() == 2 and logits.stride(1) == 1 and logits.shape[0] == S * B * R
+    rc = lib().tsd_accept_relaxed(
+        S, B, int(n_cur), R, _ptr(parent), _ptr(state), int(mask_id), _ptr(conf), _ptr(topk_idx),
+        int(topk_idx.shape[-1]) if topk_idx.dim() == 4 else 1, int(topk_m), _ptr(logits),
+        0 if logits is None else dtype_code(logits.dtype), 0 if logits is None else logits.shape[1],
+        0 if logits is None else logits.stride(0), _ptr(lse), float(tau), int(rule), int(search),
+        _ptr(edge_valid), _ptr(prefix_len), _ptr(accepted_node), _ptr(accepted_len), _ptr(n_new_tokens),
+        _ptr(unmask_flag), _ptr(unmask_tok), _ptr(draft_prob), _ptr(status), _stream(stream))
+    _check(rc, "tsd_accept_relaxed")

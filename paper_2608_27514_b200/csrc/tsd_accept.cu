@@ -6,6 +6,12 @@
 // as warp ballots over the block's rows; one thread then walks the tree (a few dozen nodes).
 // Integer and float compares only: the result is exact.
 //
+// Besides the exact and top-1 tests, the two relaxed readings of the verification test
+// ("fall within top-k / exceed tau"): membership of the drafted token in the parent's first
+// topk_m candidates, and the probability of the drafted token under the parent's distribution,
+// gathered here from the logits and the row's log-sum-exp (one scattered load per drafted token;
+// the vocabulary pass has already produced the log-sum-exp).
+//
 // The joint pass of inter-block speculation (Section 3.4) verifies two trees at once: branches
 // [0, n_cur) and [n_cur, B) of the same arrays.  blockIdx.y picks the tree; per-branch outputs
 // keep their position in the forest, per-tree outputs are tree-major ([2, batch, ...]).
@@ -20,6 +26,15 @@ constexpr int kMaxRows = 128;
 constexpr int kRowWords = kMaxRows / 32;
 constexpr int kAcceptThreads = 256;
 
+struct RelaxedArgs {
+  int topk_m;           // candidates per row that count for TSD_ACCEPT_TOPK
+  const void* logits;   // [batch, B, R, vocab] rows `ld` elements apart, nullable
+  int dtype;
+  int64_t vocab, ld;
+  const float* lse;     // [batch, B, R] natural-log sum-exp of each logits row
+  float* draft_prob;    // [batch, B, R] out, nullable
+};
+
 __global__ void __launch_bounds__(kAcceptThreads)
 accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
               int mask_id, const float* __restrict__ conf, const int32_t* __restrict__ top1,
@@ -27,7 +42,7 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
               int32_t* __restrict__ prefix_len, int32_t* __restrict__ accepted_node,
               int32_t* __restrict__ accepted_len, int32_t* __restrict__ n_new_tokens,
               uint8_t* __restrict__ unmask_flag, int32_t* __restrict__ unmask_tok,
-              uint32_t* __restrict__ status) {
+              uint32_t* __restrict__ status, RelaxedArgs x) {
   __shared__ uint32_t s_u[kMaxBranches][kRowWords];  // U(p) as a row bitset
   __shared__ uint8_t s_valid[kMaxBranches];
   __shared__ int s_par[kMaxBranches];
@@ -99,10 +114,11 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   for (int c = warp; c < B; c += n_warps) {
     const int p = s_par[c];
     bool ok = true, malformed = false, delta = false;
-    if (c > 0 && p >= 0) {
-      for (int w = 0; w < words; ++w) {
-        const int r = w * 32 + lane;
-        if (r < R) {
+    for (int w = 0; w < words; ++w) {
+      const int r = w * 32 + lane;
+      if (r < R) {
+        float pr = 0.f;  // probability of the token this child adds at r, under its parent
+        if (c > 0 && p >= 0) {
           const int sp = st[p * R + r], sc = st[c * R + r];
           const bool p_masked = sp == mask_id, c_masked = sc == mask_id;
           const bool in_u = (s_u[p][w] >> lane) & 1u;
@@ -112,10 +128,23 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
             if (rule == TSD_ACCEPT_EXACT && in_u) ok = false;  // U has a row the child lacks
           } else {
             delta = true;
-            const bool tok_ok = t1[(size_t)(p * R + r) * top1_stride] == sc;
-            if (rule == TSD_ACCEPT_EXACT) ok &= in_u && tok_ok; else ok &= tok_ok;
+            const int32_t* cand = t1 + (size_t)(p * R + r) * top1_stride;
+            bool tok_ok = cand[0] == sc;
+            if (rule == TSD_ACCEPT_TOPK)
+              for (int j = 1; j < x.topk_m; ++j) tok_ok |= cand[j] == sc;
+            if (x.logits && sc >= 0 && sc < x.vocab) {
+              const size_t row = ((size_t)s * B_all + lo + p) * R + r;
+              const float z = x.dtype == TSD_BF16
+                                  ? __bfloat162float(static_cast<const __nv_bfloat16*>(x.logits)[row * x.ld + sc])
+                                  : static_cast<const float*>(x.logits)[row * x.ld + sc];
+              pr = expf(z - x.lse[row]);
+            }
+            if (rule == TSD_ACCEPT_EXACT) ok &= in_u && tok_ok;
+            else if (rule == TSD_ACCEPT_PROB) ok &= pr > tau;  // strictly above, as in Alg. 1
+            else ok &= tok_ok;
           }
         }
+        if (x.draft_prob) x.draft_prob[((size_t)s * B_all + lo + c) * R + r] = pr;
       }
     }
     const bool all_ok = __all_sync(full, ok), any_bad = __any_sync(full, malformed),
@@ -185,11 +214,18 @@ static int accept_launch(int32_t batch, int32_t n_branches, int32_t n_cur, int32
                          const int32_t* top1_idx, int32_t top1_stride, float tau, int32_t rule,
                          int32_t search, uint8_t* edge_valid, int32_t* prefix_len, int32_t* accepted_node,
                          int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
-                         int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream) {
+                         int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream,
+                         const tsd::RelaxedArgs& x) {
   if (batch < 0 || n_cur < 1 || n_cur > n_branches || n_branches < 1 || n_branches > tsd::kMaxBranches || rows_per_branch < 1 ||
       rows_per_branch > tsd::kMaxRows || top1_stride < 1)
     return TSD_ERR_INVALID_ARG;
-  if (rule != TSD_ACCEPT_EXACT && rule != TSD_ACCEPT_TOP1) return TSD_ERR_INVALID_ARG;
+  if (rule < TSD_ACCEPT_EXACT || rule > TSD_ACCEPT_PROB) return TSD_ERR_INVALID_ARG;
+  if (rule == TSD_ACCEPT_TOPK && (x.topk_m < 1 || x.topk_m > top1_stride)) return TSD_ERR_INVALID_ARG;
+  if (rule == TSD_ACCEPT_PROB && !x.logits) return TSD_ERR_INVALID_ARG;
+  if (x.logits) {
+    if (x.dtype != TSD_F32 && x.dtype != TSD_BF16) return TSD_ERR_UNSUPPORTED;
+    if (!x.lse || x.vocab < 1 || x.ld < x.vocab) return TSD_ERR_INVALID_ARG;
+  }
   if (search != TSD_SEARCH_GREEDY && search != TSD_SEARCH_LONGEST) return TSD_ERR_INVALID_ARG;
   if (!(tau == tau)) return TSD_ERR_INVALID_ARG;  // NaN threshold
   if (batch == 0) return TSD_OK;
@@ -200,7 +236,7 @@ static int accept_launch(int32_t batch, int32_t n_branches, int32_t n_cur, int32
   tsd::accept_kernel<<<grid, tsd::kAcceptThreads, 0, stream>>>(
       n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
       search, edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
-      unmask_tok, status);
+      unmask_tok, status, x);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return tsd::cuda_fail(e, "accept_kernel");
   return TSD_OK;
@@ -214,9 +250,10 @@ extern "C" int tsd_accept_trajectories(int32_t batch, int32_t n_branches, int32_
                                        int32_t* accepted_len, int32_t* n_new_tokens,
                                        uint8_t* unmask_flag, int32_t* unmask_tok, uint32_t* status,
                                        tsd_stream_t stream) {
+  if (rule != TSD_ACCEPT_EXACT && rule != TSD_ACCEPT_TOP1) return TSD_ERR_INVALID_ARG;
   return accept_launch(batch, n_branches, n_branches, rows_per_branch, parent, state, mask_id, conf, top1_idx,
                        top1_stride, tau, rule, search, edge_valid, prefix_len, accepted_node, accepted_len,
-                       n_new_tokens, unmask_flag, unmask_tok, status, stream);
+                       n_new_tokens, unmask_flag, unmask_tok, status, stream, tsd::RelaxedArgs{});
 }
 
 extern "C" int tsd_accept_joint_trees(int32_t batch, int32_t n_branches, int32_t n_cur,
@@ -226,7 +263,30 @@ extern "C" int tsd_accept_joint_trees(int32_t batch, int32_t n_branches, int32_t
                                       uint8_t* edge_valid, int32_t* prefix_len, int32_t* accepted_node,
                                       int32_t* accepted_len, int32_t* n_new_tokens, uint8_t* unmask_flag,
                                       int32_t* unmask_tok, uint32_t* status, tsd_stream_t stream) {
+  if (rule != TSD_ACCEPT_EXACT && rule != TSD_ACCEPT_TOP1) return TSD_ERR_INVALID_ARG;
   return accept_launch(batch, n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx,
                        top1_stride, tau, rule, search, edge_valid, prefix_len, accepted_node, accepted_len,
-                       n_new_tokens, unmask_flag, unmask_tok, status, stream);
+                       n_new_tokens, unmask_flag, unmask_tok, status, stream, tsd::RelaxedArgs{});
+}
+
+extern "C" int tsd_accept_relaxed(int32_t batch, int32_t n_branches, int32_t n_cur, int32_t rows_per_branch,
+                                  const int32_t* parent, const int32_t* state, int32_t mask_id,
+                                  const float* conf, const int32_t* topk_idx, int32_t topk_stride,
+                                  int32_t topk_m, const void* logits, int32_t dtype, int64_t vocab,
+                                  int64_t row_stride, const float* lse, float tau, int32_t rule,
+                                  int32_t search, uint8_t* edge_valid, int32_t* prefix_len,
+                                  int32_t* accepted_node, int32_t* accepted_len, int32_t* n_new_tokens,
+                                  uint8_t* unmask_flag, int32_t* unmask_tok, float* draft_prob,
+                                  uint32_t* status, tsd_stream_t stream) {
+  tsd::RelaxedArgs x{};
+  x.topk_m = topk_m;
+  x.logits = logits;
+  x.dtype = dtype;
+  x.vocab = vocab;
+  x.ld = row_stride;
+  x.lse = lse;
+  x.draft_prob = logits ? draft_prob : nullptr;
+  return accept_launch(batch, n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, topk_idx,
+                       topk_stride, tau, rule, search, edge_valid, prefix_len, accepted_node, accepted_len,
+                       n_new_tokens, unmask_flag, unmask_tok, status, stream, x);
 }

@@ -71,6 +71,20 @@ class VerifyStep:
             self.n_new_tokens, self.unmask_flag, self.unmask_tok, self.status)
         return self.accept_outputs()
 
+    def accept_relaxed(self, parent, state, mask_id, tau, rule, search=B.TSD_SEARCH_LONGEST, logits=None,
+                       topk_m=None):
+        """Acceptance under any rule, on the candidates and log-sum-exp of the last vocabulary pass;
+        the probability rule gathers from `logits` (the tensor that pass read)."""
+        if logits is not None and not hasattr(self, "draft_prob"):
+            self.draft_prob = torch.empty((self.S, self.B, self.R), dtype=torch.float32, device=self.device)
+        B.tsd_accept_relaxed(
+            parent, state, self.B, mask_id, self.conf, self.topk_idx.view(self.S, self.B, self.R, self.k),
+            self.k if topk_m is None else topk_m, logits, self.lse if logits is not None else None, tau, rule,
+            search, self.edge_valid, self.prefix_len, self.accepted_node, self.accepted_len, self.n_new_tokens,
+            self.unmask_flag, self.unmask_tok, getattr(self, "draft_prob", None) if logits is not None else None,
+            self.status)
+        return self.accept_outputs()
+
     def accept_outputs(self):
         return dict(edge_valid=self.edge_valid, prefix_len=self.prefix_len,
                     accepted_node=self.accepted_node, accepted_len=self.accepted_len,

@@ -156,3 +156,23 @@ def test_interblock_validation(lib):
     assert call(n_cur=9) == B.TSD_ERR_INVALID_ARG
     assert call(R=129) == B.TSD_ERR_INVALID_ARG
     assert call(rule=2) == B.TSD_ERR_INVALID_ARG
+
+
+def test_relaxed_accept_validation(lib):
+    p = ctypes.c_void_p(4096)
+    f = lib.tsd_accept_relaxed
+
+    def call(rule=2, stride=3, m=2, logits=None, dtype=1, vocab=100, ld=100, lse=p, R=32, n_cur=4):
+        return f(1, 4, n_cur, R, p, p, 99, p, p, stride, m, logits, dtype, vocab, ld, lse, 0.9, rule, 0,
+                 *([p] * 7), None, None, None)
+    assert call(m=4) == B.TSD_ERR_INVALID_ARG                 # more candidates than the list holds
+    assert call(m=0) == B.TSD_ERR_INVALID_ARG
+    assert call(rule=3) == B.TSD_ERR_INVALID_ARG              # the probability rule needs logits
+    assert call(rule=4) == B.TSD_ERR_INVALID_ARG
+    assert call(rule=3, logits=p, lse=None) == B.TSD_ERR_INVALID_ARG
+    assert call(rule=3, logits=p, ld=99) == B.TSD_ERR_INVALID_ARG
+    assert call(rule=3, logits=p, dtype=5) == B.TSD_ERR_UNSUPPORTED
+    assert call(n_cur=5) == B.TSD_ERR_INVALID_ARG
+    # the strict entry points do not take the relaxed rules
+    assert lib.tsd_accept_trajectories(1, 4, 32, p, p, 99, p, p, 1, 0.9, 2, 0, *([p] * 7), None, None) \
+        == B.TSD_ERR_INVALID_ARG

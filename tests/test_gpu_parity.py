@@ -250,7 +250,7 @@ def _gpu_accept(parent, state, mask_id, conf, top1, tau, rule, search, stride=1)
     return {k: v.cpu().numpy() for k, v in out.items()}, status
 
 
-CASES = load_accept_cases()
+CASES = [c for c in load_accept_cases() if c["rule"] <= 1]   # the relaxed rules: test_gpu_relaxed.py
 
 
 @pytest.mark.parametrize("case", CASES, ids=[c["id"] for c in CASES])
