@@ -6,7 +6,8 @@ tests, the smoke check and the benchmark's CPU-baseline leg may import this
 package; the CUDA library never does, and the two share no code.
 
 ``theorem1`` holds the toy-model harness for the exactness theorem; ``interblock`` the joint
-mask, trigger and two-tree acceptance of inter-block speculation (Section 3.4).
+mask, trigger and two-tree acceptance of inter-block speculation (Section 3.4); ``commit`` the
+bookkeeping that turns an accepted path into the next root and its sequential step indices.
 """
 from .binding import (  # noqa: F401
     build,
