@@ -73,6 +73,7 @@ typedef enum { TSD_SEARCH_GREEDY = 0, TSD_SEARCH_LONGEST = 1 } tsd_search;
 #define TSD_STATUS_TIMEOUT 0x1u     /* a bounded wait inside a kernel expired      */
 #define TSD_STATUS_BAD_PARENT 0x2u  /* parent[b] outside [0, b) for some b > 0     */
 #define TSD_STATUS_BAD_MASK 0x4u    /* mask blob header does not match the layout  */
+#define TSD_STATUS_BAD_INDEX 0x8u   /* a position read from device memory is out of range */
 
 /* tsd_verify_attention flags */
 #define TSD_ATTN_FORCE_SIMT 0x1u /* use the CUDA-core kernel even where the tensor-core one applies */
@@ -313,6 +314,40 @@ int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_t rows_per_
  * ------------------------------------------------------------------------- */
 int tsd_build_interblock_vis(int32_t batch, int32_t n_branches, int32_t n_cur, uint64_t* vis,
                              tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * The step after the path: commit what the pass accepted (Section 3.3: the
+ * longest verified trajectory is kept; Section 3.1: its last node starts the
+ * next pass; Theorem 1: each edge of the accepted path is one step of the
+ * sequential decoder).  Per sequence: next root = state of the accepted node +
+ * its unmask set, written to root_out and into the sequence's token buffer at
+ * the block's position.  With the pass starting step_base sequential steps into
+ * the block and accepting a node of depth n, a row filled by the path node at
+ * depth j is logged at step step_base + j - 1, the rows of the unmask set at
+ * step_base + n, and step_base moves on by n + 1 (by n if the accepted node had
+ * no masked row left).
+ *
+ *   parent, state   device [batch, B] / [batch, B, R]: the verified tree;
+ *   accepted_node   device int32 [batch], nullable (= node 0);
+ *   unmask_flag, unmask_tok   device [batch, R], both or neither;
+ *   tokens          device int32, nullable: sequence s occupies tokens[s * seq_stride ...];
+ *   block_start     device int32 [batch], nullable (= 0): first position of the block; a
+ *                   block that does not fit in [0, seq_stride) sets TSD_STATUS_BAD_INDEX and
+ *                   is not written;
+ *   root_out        device int32 [batch, R], nullable;
+ *   fill_step       device int32 [batch, R], nullable, in/out: only rows filled by this pass
+ *                   are written (initialise with -1 at the start of a block);
+ *   step_base       device int32 [batch], nullable (= 0), in/out;
+ *   n_masked        device int32 [batch], nullable: rows still masked in the next root.
+ * A parent chain that leaves the tree sets TSD_STATUS_BAD_PARENT and commits U(root) only.
+ * R 1..128, B 1..256.
+ * ------------------------------------------------------------------------- */
+int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+                        const int32_t* parent, const int32_t* state, const int32_t* accepted_node,
+                        const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
+                        int32_t* tokens, int64_t seq_stride, const int32_t* block_start,
+                        int32_t* root_out, int32_t* fill_step, int32_t* step_base, int32_t* n_masked,
+                        uint32_t* status, tsd_stream_t stream);
 
 /* ---------------------------------------------------------------------------
  * Acceptance under any of the four rules (Section 3.3, "Verification

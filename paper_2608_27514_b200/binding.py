@@ -28,6 +28,7 @@ EXPORTS = (
     "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
     "tsd_accept_trajectories", "tsd_build_draft_tree",
     "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees", "tsd_accept_relaxed",
+    "tsd_commit_accepted",
 )
 
 
@@ -89,6 +90,8 @@ def lib():
                                              _i32, _i32] + [_vp] * 9
         L.tsd_accept_relaxed.argtypes = ([_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _vp, _i32,
                                           _i64, _i64, _vp, _f32, _i32, _i32] + [_vp] * 10)
+        L.tsd_commit_accepted.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _vp, _vp,
+                                          _vp, _vp, _vp, _vp, _vp]
         _lib = L
     return _lib
 
@@ -283,3 +286,17 @@ def tsd_accept_relaxed(parent, state, n_cur, mask_id, conf, topk_idx, topk_m, lo
         _ptr(edge_valid), _ptr(prefix_len), _ptr(accepted_node), _ptr(accepted_len), _ptr(n_new_tokens),
         _ptr(unmask_flag), _ptr(unmask_tok), _ptr(draft_prob), _ptr(status), _stream(stream))
     _check(rc, "tsd_accept_relaxed")
+
+
+def tsd_commit_accepted(parent, state, accepted_node, unmask_flag, unmask_tok, mask_id, tokens=None,
+                        block_start=None, root_out=None, fill_step=None, step_base=None, n_masked=None,
+                        status=None, stream=None):
+    """parent [S,B], state [S,B,R]; tokens [S,L] (row stride = tokens.stride(0)); the rest [S] / [S,R]."""
+    S, B, R = state.shape
+    if tokens is not None:
+        assert tokens.dim() == 2 and tokens.stride(1) == 1
+    rc = lib().tsd_commit_accepted(
+        S, B, R, _ptr(parent), _ptr(state), _ptr(accepted_node), _ptr(unmask_flag), _ptr(unmask_tok),
+        int(mask_id), _ptr(tokens), 0 if tokens is None else tokens.stride(0), _ptr(block_start), _ptr(root_out),
+        _ptr(fill_step), _ptr(step_base), _ptr(n_masked), _ptr(status), _stream(stream))
+    _check(rc, "tsd_commit_accepted")

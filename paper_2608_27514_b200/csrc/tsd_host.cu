@@ -46,7 +46,7 @@ const char* tsd_last_cuda_error(void) { return tsd::g_last_cuda_error; }
 
 int tsd_check_status(uint32_t w) {
   if (w & TSD_STATUS_TIMEOUT) return TSD_ERR_TIMEOUT;
-  if (w & (TSD_STATUS_BAD_PARENT | TSD_STATUS_BAD_MASK)) return TSD_ERR_DEVICE_DATA;
+  if (w & (TSD_STATUS_BAD_PARENT | TSD_STATUS_BAD_MASK | TSD_STATUS_BAD_INDEX)) return TSD_ERR_DEVICE_DATA;
   return TSD_OK;
 }
 
