@@ -49,6 +49,10 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return r;
 }
 
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
   uint32_t r;
   asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -229,7 +233,7 @@ __global__ void __launch_bounds__(THREADS)
 confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stride, int k, int n_seg,
                        int chunks_per_seg, float* __restrict__ conf, int32_t* __restrict__ topk_idx,
                        float* __restrict__ topk_prob, float* __restrict__ lse,
-                       Partial<K>* __restrict__ partials, unsigned* __restrict__ tickets) {
+                       Partial<K>* __restrict__ partials, unsigned* __restrict__ tickets, int prefetch) {
   constexpr int E = Unpack<T>::kElems;
   constexpr int kTopkThreads = THREADS, kTopkWarps = THREADS / 32;
   constexpr int kTopkBatch = THREADS * kTopkUnroll;        // chunks per block per batch
@@ -275,11 +279,20 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     for (int u = 0; u < kTopkUnroll; ++u) part[u] = Unpack<T>::sum_exp(buf[u], -e, 0.f);
     s += (part[0] + part[1]) + (part[2] + part[3]);
   };
+  // Optional L2 prefetch `prefetch` batches ahead of the register loads, one 128-byte line per
+  // thread (the launcher turns it on for large grids only).
+  auto prefetch_batch = [&](int it) {
+    constexpr int kLines = kTopkBatch * 16 / 128;  // lines per batch (<= THREADS)
+    const int c = c0 + it * kTopkBatch + tid * 8;  // first chunk of this thread's line
+    if (tid < kLines && it < n_iter && c < c1) prefetch_l2(rowv + c);
+  };
   {
     uint4 buf_a[kTopkUnroll], buf_b[kTopkUnroll];
     if (n_iter > 0) load_batch(buf_a, 0);
+    for (int p = 1; p <= prefetch; ++p) prefetch_batch(p);
     for (int it = 0; it < n_iter; it += 2) {
       if (it + 1 < n_iter) load_batch(buf_b, it + 1);
+      if (prefetch) { prefetch_batch(it + prefetch + 1); prefetch_batch(it + prefetch + 2); }
       process_batch(buf_a, it);
       if (it + 1 < n_iter) {
         if (it + 2 < n_iter) load_batch(buf_a, it + 2);
@@ -338,17 +351,21 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   a.seen = m != -CUDART_INF_F;
   a.e = e;
   a.s = s;
+  // The whole block waits for its slowest warp here, so a hit batch (32 values for bf16, 16 for
+  // fp32) is examined by the warp together: lane l re-reads value l of the batch (an L2 hit) and
+  // offers it to its own list; warp_merge combines the lanes' lists afterwards.
   for (int it = 0; it < n_iter; ++it) {
-    if (!(s_bmax[it][tid] >= bound)) continue;
-#pragma unroll 1
-    for (int u = 0; u < kTopkUnroll; ++u) {
-      const int c = c0 + it * kTopkBatch + tid + u * kTopkThreads;
-      if (c >= c1) break;
-      const uint4 w = rowv[c];
-#pragma unroll 1
-      for (int j = 0; j < E; ++j) {
-        const float x = Unpack<T>::elem(w, j);
-        if (x >= bound) a.offer(x, c * E + j);
+    unsigned hits = __ballot_sync(0xffffffffu, s_bmax[it][tid] >= bound);
+    while (hits) {
+      const int src = __ffs(hits) - 1;
+      hits &= hits - 1;
+      if (lane < kTopkUnroll * E) {
+        const int c = c0 + it * kTopkBatch + (warp * 32 + src) + (lane / E) * kTopkThreads;
+        if (c < c1) {
+          const int xi = c * E + lane % E;
+          const float x = to_float(rowp[xi]);
+          if (x >= bound) a.offer(x, xi);
+        }
       }
     }
   }
@@ -410,7 +427,7 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
 }
 
 struct TopkPlan {
-  int n_seg, chunks_per_seg, K, threads;
+  int n_seg, chunks_per_seg, K, threads, prefetch;
   size_t partial_bytes, ticket_off, total_bytes;
 };
 
@@ -431,6 +448,9 @@ static TopkPlan topk_plan(int64_t n_rows, int vocab, int k, int elems_per_chunk)
   p.n_seg = (int)std::max<int64_t>(n_seg, 1);
   // up to two 512-thread blocks fit an SM: use them while that still gives every block a slot at once
   p.threads = (n_rows * p.n_seg <= 2 * 148) ? 512 : 256;
+  // L2 prefetch distance in batches (measured): with several waves of blocks, requesting lines
+  // three batches ahead adds 3 % of bandwidth; with few blocks it only delays the demand loads
+  p.prefetch = (n_rows * p.n_seg >= 2048) ? 3 : 0;
   p.chunks_per_seg = (chunks + p.n_seg - 1) / p.n_seg;
   if (p.chunks_per_seg == 0) p.chunks_per_seg = 1;
   const size_t rec = 8 + 8 * (size_t)p.K;
@@ -453,11 +473,11 @@ static cudaError_t launch_topk(const void* logits, int64_t n_rows, int vocab, in
   if (p.threads == 512)
     confidence_topk_kernel<T, K, 512><<<(unsigned)(n_rows * p.n_seg), 512, 0, st>>>(
         static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
-        lse, partials, tickets);
+        lse, partials, tickets, p.prefetch);
   else
     confidence_topk_kernel<T, K, 256><<<(unsigned)(n_rows * p.n_seg), 256, 0, st>>>(
         static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
-        lse, partials, tickets);
+        lse, partials, tickets, p.prefetch);
   return cudaGetLastError();
 }
 
