@@ -53,6 +53,29 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
+// packed pairs of fp32 (one instruction for two lanes of arithmetic)
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
   uint32_t r;
   asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -213,16 +236,21 @@ struct Unpack<__nv_bfloat16> {
     return __uint_as_float((j & 1) ? (word & 0xffff0000u) : (word << 16));
   }
   static __device__ __forceinline__ float sum_exp(const uint4& w, float ne, float s) {
-    // two partial sums per chunk keep the dependent add chain short
-    float s1 = ex2_approx(fmaf(__uint_as_float(w.x & 0xffff0000u), kLog2e, ne));
-    s += ex2_approx(fmaf(__uint_as_float(w.x << 16), kLog2e, ne));
-    s1 += ex2_approx(fmaf(__uint_as_float(w.y & 0xffff0000u), kLog2e, ne));
-    s += ex2_approx(fmaf(__uint_as_float(w.y << 16), kLog2e, ne));
-    s1 += ex2_approx(fmaf(__uint_as_float(w.z & 0xffff0000u), kLog2e, ne));
-    s += ex2_approx(fmaf(__uint_as_float(w.z << 16), kLog2e, ne));
-    s1 += ex2_approx(fmaf(__uint_as_float(w.w & 0xffff0000u), kLog2e, ne));
-    s += ex2_approx(fmaf(__uint_as_float(w.w << 16), kLog2e, ne));
-    return s + s1;
+    // a bf16 pair widens to an fp32 pair with one shift and one mask; the scale-and-shift and the
+    // accumulation run as packed fp32 pairs, only the exponentials are per value
+    const uint64_t l2 = pack2(__float_as_uint(kLog2e), __float_as_uint(kLog2e));
+    const uint64_t ne2 = pack2(__float_as_uint(ne), __float_as_uint(ne));
+    uint64_t acc = pack2(0u, 0u);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float t0, t1;
+      unpack2(fma2(pack2(words[q] << 16, words[q] & 0xffff0000u), l2, ne2), t0, t1);
+      acc = add2(acc, pack2(__float_as_uint(ex2_approx(t0)), __float_as_uint(ex2_approx(t1))));
+    }
+    float a0, a1;
+    unpack2(acc, a0, a1);
+    return s + (a0 + a1);
   }
 };
 
