@@ -237,6 +237,7 @@ struct TcParams {
   uint32_t* status;
   int64_t os_b, os_r, os_h;
   int S, B, R, Nc, N, Hq, group;
+  int recs_off, n_qt, rec_words;  // layout of the mask blob, computed on the host from the same tsd_layout
   float scale_log2e;  // sm_scale * log2(e), > 0
 };
 
@@ -256,20 +257,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int g = h / p.group;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  // Everything the block needs from the mask blob is requested at once (the blob's layout follows
+  // from the tsd_layout, so no address depends on a loaded value); the producer thread meanwhile
+  // sets up the barriers and starts the Q load, so the two latencies overlap.
   const int32_t* mask = p.mask;
-  const bool hdr_ok = mask[H_MAGIC] == kMaskMagic && mask[H_S] == p.S && mask[H_B] == p.B &&
-                      mask[H_R] == p.R && mask[H_NC] == p.Nc;
-  if (!hdr_ok) {  // uniform over the block: nothing has been set up yet
-    if (tid == 0 && p.status) atomicOr(p.status, TSD_STATUS_BAD_MASK);
-    return;
-  }
+  const int32_t* rec = mask + p.recs_off + (size_t)(s * p.n_qt + qt) * p.rec_words;
+  const int h_magic = mask[H_MAGIC], h_s = mask[H_S], h_b = mask[H_B], h_r = mask[H_R], h_nc = mask[H_NC];
   const int clen = mask[kHdrWords + s];
-  const int32_t* rec = mask + mask[H_RECS_OFF] + (size_t)(s * mask[H_NQT] + qt) * mask[H_REC_WORDS];
-  const int n_ct = (clen + kKeys - 1) / kKeys;  // cached tiles of 64 keys
-  const int n_dt = rec[0];                      // visible 128-row draft tiles = 2 key tiles each
-  const int T = n_ct + 2 * n_dt;
+  const int n_dt_raw = rec[0];  // visible 128-row draft tiles = 2 key tiles each
 
-  if (tid == 0) {
+  if (warp == 4 && lane == 0) {
     abort_flag[0] = 0;
     abort_flag[1] = 0;  // scratch flag for the producer's drain waits
     mbar_init(bar(Q_FULL), 1);
@@ -282,11 +279,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
+    mbar_expect_tx(bar(Q_FULL), kTileBytes);
+    tma_load_4d(base + kOffQ, &map_q, bar(Q_FULL), 0, h, qt * kTile, s);
+    tma_load_4d(base + kOffQ + kSub, &map_q, bar(Q_FULL), 64, h, qt * kTile, s);
   }
   if (warp == 5) {  // TMEM: 2 x S/P (64 columns each) + O (128 columns); two blocks share the SM's 512
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(bars + 128u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // A blob that was built for another layout: report it and run the block with no key tiles and
+  // no output (the Q load in flight is still waited for before the block leaves).
+  const bool hdr_ok = h_magic == kMaskMagic && h_s == p.S && h_b == p.B && h_r == p.R && h_nc == p.Nc;
+  if (!hdr_ok && tid == 0 && p.status) atomicOr(p.status, TSD_STATUS_BAD_MASK);
+  const int n_ct = hdr_ok ? (clen + kKeys - 1) / kKeys : 0;  // cached tiles of 64 keys
+  const int n_dt = hdr_ok ? n_dt_raw : 0;
+  const int T = n_ct + 2 * n_dt;
+
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -304,9 +312,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tma_load_4d(dst, m, full_bar, 0, g, row, s);
         tma_load_4d(dst + kSubKV, m, full_bar, 64, g, row, s);
       };
-      mbar_expect_tx(bar(Q_FULL), kTileBytes);
-      tma_load_4d(base + kOffQ, &map_q, bar(Q_FULL), 0, h, qt * kTile, s);
-      tma_load_4d(base + kOffQ + kSub, &map_q, bar(Q_FULL), 64, h, qt * kTile, s);
       bool ok = true;
       int k_issued = 0, v_issued = 0;
       auto load_k = [&](int j) {
@@ -517,7 +522,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     // epilogue: O / l -> bf16 -> global, lse
     if (ok && T > 0) ok = mbar_wait(bar(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag);
-    if (ok) {
+    if (ok && hdr_ok) {
       tc_fence_after();
       const int i = qt * kTile + r;
       const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -640,6 +645,8 @@ int launch_attention_tc(const AttnArgs& a) {
   p.os_b = a.os_b; p.os_r = a.os_r; p.os_h = a.os_h;
   p.S = L.batch; p.B = L.n_branches; p.R = L.rows_per_branch; p.Nc = L.n_cache; p.N = N;
   p.Hq = L.n_q_heads; p.group = L.n_q_heads / L.n_kv_heads;
+  const MaskDims md = mask_dims(L);
+  p.recs_off = md.recs_off; p.n_qt = md.n_qt; p.rec_words = md.rec_words;
   p.scale_log2e = a.sm_scale * kLog2e;
   dim3 grid((N + kTile - 1) / kTile, L.n_q_heads, L.batch);
   attention_tc_kernel<<<grid, kTcThreads, kSmemBytes, a.stream>>>(mq, mkc, mvc, mkd, mvd, p);

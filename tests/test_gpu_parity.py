@@ -68,6 +68,22 @@ def _check_attention(cfg, attn, flags, vis=None, cache_lens=None, heads=None, se
 
 
 # ----------------------------------------------------------------------------- mask
+@pytest.mark.parametrize("flags", PATHS)
+def test_attention_reports_a_mask_built_for_another_layout(flags):
+    cfg = W.small(W.CONFIGS["cfg2"], S=1, B=4, R=32, Nc=64, Hq=2, Hkv=2)
+    other = VerifyStep.for_config(W.small(cfg, B=8), DEV)
+    other.build_mask()                                  # a (larger) blob for 8 branches
+    step = VerifyStep.for_config(cfg, DEV)
+    step.mask, step.mask_built = other.mask, True
+    step.out.fill_(7.0)
+    attn = W.attention_inputs(cfg, DEV)
+    step.attention(attn["q"], attn["k_cache"], attn["v_cache"], attn["k_draft"], attn["v_draft"], attn["sm_scale"],
+                   flags)
+    torch.cuda.synchronize()
+    assert B.tsd_check_status(step.status) == B.TSD_ERR_DEVICE_DATA
+    assert (step.out == 7.0).all()                      # nothing was written
+
+
 def test_mask_dense_matches_oracle_with_vis_and_ragged_cache():
     cfg = W.small(W.CONFIGS["cfg2"], S=3, B=9, Nc=100, Hq=1, Hkv=1)
     rng = np.random.default_rng(0)
