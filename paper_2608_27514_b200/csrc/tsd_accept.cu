@@ -46,6 +46,8 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   __shared__ uint32_t s_u[kMaxBranches][kRowWords];  // U(p) as a row bitset
   __shared__ uint8_t s_valid[kMaxBranches];
   __shared__ int s_par[kMaxBranches];
+  __shared__ int s_pl[kMaxBranches];  // prefix_len, kept on chip for the walk (global reads of values
+                                      // just written would cost one L2 round trip per node)
   __shared__ int s_acc;
   const int s = blockIdx.x, tree = blockIdx.y, batch = gridDim.x;
   const int lo = tree ? n_cur : 0;          // first branch of this tree = its root
@@ -73,6 +75,7 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
         if (r < R) {
           masked = st[p * R + r] == mask_id;
           const float c = cf[p * R + r];
+
           high = masked && c > tau;  // strictly above the threshold
           if (masked && (best_r == INT_MAX || c > best)) { best = c; best_r = r; }  // rows ascend
         }
@@ -155,11 +158,11 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
 
   // tree walk (parents precede children, so one ascending sweep fills depth and prefix length)
   if (threadIdx.x == 0) {
-    // prefix_len is read back from the global array this block has just written; a node's depth
-    // is found by walking its parents (trees are a few levels deep)
+    // a node's depth is found by walking its parents (trees are a few levels deep)
     int32_t* pl = prefix_len + (size_t)s * B_all + lo;
     uint8_t* ev = edge_valid + (size_t)s * B_all + lo;
     int acc = 0, acc_depth = 0;
+    s_pl[0] = 0;
     pl[0] = 0;
     ev[0] = 1;
     for (int b = 1; b < B; ++b) {
@@ -167,9 +170,11 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
       ev[b] = s_valid[b];
       int depth_p = 0;
       for (int a = p; a > 0; a = s_par[a]) ++depth_p;
-      const int plp = p >= 0 ? pl[p] : 0;
+      const int plp = p >= 0 ? s_pl[p] : 0;
       const bool whole = p >= 0 && plp == depth_p && s_valid[b];
-      pl[b] = whole ? depth_p + 1 : plp;
+      const int plb = whole ? depth_p + 1 : plp;
+      s_pl[b] = plb;
+      pl[b] = plb;
       if (search == TSD_SEARCH_LONGEST && whole && depth_p + 1 > acc_depth) { acc = b; acc_depth = depth_p + 1; }
     }
     if (search == TSD_SEARCH_GREEDY) {
