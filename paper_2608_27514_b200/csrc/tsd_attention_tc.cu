@@ -95,6 +95,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
 // True in exactly one lane of a converged warp; the compiler recognises the pattern and keeps the
 // warp's address arithmetic on the uniform datapath, which the tcgen05 instructions read.
 __device__ __forceinline__ bool elect_one() {
@@ -244,7 +249,8 @@ struct TcParams {
 __global__ void __launch_bounds__(kTcThreads, 2)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                     const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kd,
-                    const __grid_constant__ CUtensorMap map_vd, const TcParams p) {
+                    const __grid_constant__ CUtensorMap map_vd, const __grid_constant__ CUtensorMap map_o,
+                    const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -523,10 +529,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // epilogue: O / l -> bf16 -> global, lse
     if (ok && T > 0) ok = mbar_wait(bar(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag);
     if (ok && hdr_ok) {
+      // O / l -> bf16 -> the shared memory that held Q (every Q K^T has completed), in the layout
+      // of the output tensor map (128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)),
+      // then one TMA store per half of head_dim: full 128-byte rows instead of 16-byte pieces per
+      // thread, and rows past the end of the tensor are clipped by the copy engine.
       tc_fence_after();
       const int i = qt * kTile + r;
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* orow = p.out + s * p.os_b + (int64_t)i * p.os_r + h * p.os_h;
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t ov[32];
@@ -537,19 +546,30 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
           for (int x = 0; x < 32; ++x) ov[x] = 0u;
         }
-        if (i < p.N) {
+        const uint32_t row_base = base + kOffQ + (q4 >> 1) * kSub + (uint32_t)r * 128u;
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(ov[8 * x + 0]) * inv, __uint_as_float(ov[8 * x + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(ov[8 * x + 2]) * inv, __uint_as_float(ov[8 * x + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(ov[8 * x + 4]) * inv, __uint_as_float(ov[8 * x + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(ov[8 * x + 6]) * inv, __uint_as_float(ov[8 * x + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + q4 * 32 + x * 8) = w;
-          }
+        for (int x = 0; x < 4; ++x) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(ov[8 * x + 0]) * inv, __uint_as_float(ov[8 * x + 1]) * inv);
+          w.y = pack_bf16x2(__uint_as_float(ov[8 * x + 2]) * inv, __uint_as_float(ov[8 * x + 3]) * inv);
+          w.z = pack_bf16x2(__uint_as_float(ov[8 * x + 4]) * inv, __uint_as_float(ov[8 * x + 5]) * inv);
+          w.w = pack_bf16x2(__uint_as_float(ov[8 * x + 6]) * inv, __uint_as_float(ov[8 * x + 7]) * inv);
+          const uint32_t chunk = (uint32_t)((q4 & 1) * 4 + x) ^ ((uint32_t)r & 7u);
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(row_base + (chunk << 4)), "r"(w.x), "r"(w.y),
+                       "r"(w.z), "r"(w.w) : "memory");
         }
       }
       if (p.lse && i < p.N) p.lse[((size_t)s * p.Hq + h) * p.N + i] = (m_used + log2f(l)) * kLn2;
+      fence_async_smem();
+    }
+    // the four softmax warps meet (named barrier 1; every thread of them arrives, also after a
+    // timeout), then one thread hands the tile to the copy engine and waits until it has been read
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (tid == 0 && ok && hdr_ok && !*abort_flag) {
+      tma_store_4d(&map_o, base + kOffQ, 0, h, qt * kTile, s);
+      tma_store_4d(&map_o, base + kOffQ + kSub, 64, h, qt * kTile, s);
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     }
   }
 
@@ -619,8 +639,9 @@ size_t attention_tc_workspace_bytes(const tsd_layout&) { return 0; }
 int launch_attention_tc(const AttnArgs& a) {
   const tsd_layout& L = a.L;
   const int N = L.n_branches * L.rows_per_branch;
-  CUtensorMap mq, mkc, mvc, mkd, mvd;
+  CUtensorMap mq, mkc, mvc, mkd, mvd, mo;
   bool ok = make_map(&mq, a.q, L.batch, N, L.n_q_heads, a.qs_b, a.qs_r, a.qs_h, kTile) &&
+            make_map(&mo, a.out, L.batch, N, L.n_q_heads, a.os_b, a.os_r, a.os_h, kTile) &&
             make_map(&mkd, a.kd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h, kKeys) &&
             make_map(&mvd, a.vd, L.batch, N, L.n_kv_heads, a.ds_b, a.ds_r, a.ds_h, kKeys);
   if (ok && L.n_cache > 0) {
@@ -649,7 +670,7 @@ int launch_attention_tc(const AttnArgs& a) {
   p.recs_off = md.recs_off; p.n_qt = md.n_qt; p.rec_words = md.rec_words;
   p.scale_log2e = a.sm_scale * kLog2e;
   dim3 grid((N + kTile - 1) / kTile, L.n_q_heads, L.batch);
-  attention_tc_kernel<<<grid, kTcThreads, kSmemBytes, a.stream>>>(mq, mkc, mvc, mkd, mvd, p);
+  attention_tc_kernel<<<grid, kTcThreads, kSmemBytes, a.stream>>>(mq, mkc, mvc, mkd, mvd, mo, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "attention_tc_kernel");
   return TSD_OK;
