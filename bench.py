@@ -483,7 +483,12 @@ def main():
         e2e=dict(value=world * cfg.rows / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(h2d),
                  d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms),
         gpu_launches=launches_per_step * args.steps,
-        roofline=roof, stages=stages, cpu_baseline=cpu)
+        roofline=roof, stages=stages, cpu_baseline=cpu,
+        # secondary line: a 32-layer model runs the attention stage once per layer and the vocabulary
+        # pass and the acceptance once per step; from the per-stage timings above
+        secondary=dict(metric="verified draft-token rows per second with 32 attention layers per step",
+                       value=world * cfg.rows / (32 * t_attn + t_topk + t_acc), unit=UNIT,
+                       attention_layers_per_step=32))
     print(json.dumps(line))
     replicas.shutdown()
 
