@@ -7,7 +7,8 @@ package; the CUDA library never does, and the two share no code.
 
 ``theorem1`` holds the toy-model harness for the exactness theorem; ``interblock`` the joint
 mask, trigger and two-tree acceptance of inter-block speculation (Section 3.4); ``commit`` the
-bookkeeping that turns an accepted path into the next root and its sequential step indices.
+bookkeeping that turns an accepted path into the next root and its sequential step indices;
+``fp8`` the e4m3 decode and dequantisation of the FP8 K/V cache variant.
 """
 from .binding import (  # noqa: F401
     build,
