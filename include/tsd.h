@@ -159,6 +159,35 @@ int tsd_verify_attention(const tsd_layout* layout, const void* mask,
                          uint32_t flags, uint32_t* status, tsd_stream_t stream);
 
 /* ---------------------------------------------------------------------------
+ * Verify attention over an 8-bit K/V cache.  No counterpart in the paper, which
+ * keeps the dual cache in the model's dtype: the cache is stored as e4m3 codes
+ * (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) with one
+ * fp32 scale per (sequence, kv head), half the footprint of bf16.  A cached
+ * value is bf16(decode(code) * scale) (product and rounding in fp32 -> bf16);
+ * the call expands both caches into the workspace with a streaming kernel and
+ * then runs tsd_verify_attention on the expanded copy, so results equal that
+ * call on the dequantised cache bit for bit.  Arguments as for
+ * tsd_verify_attention, except
+ *   k_cache_e4m3, v_cache_e4m3   device uint8 [batch, n_cache, n_kv_heads, head_dim], strides
+ *                c_* in elements (= bytes), multiples of 16, head_dim contiguous;
+ *   k_scale, v_scale             device fp32 [batch, n_kv_heads], nullable (= 1);
+ *   workspace    tsd_verify_attention_fp8_cache_workspace_bytes() bytes, 16-byte aligned; it is
+ *                scratch (can be shared by all layers), the persistent cache stays 8-bit.
+ * Only for layout dtype TSD_BF16 (else TSD_ERR_UNSUPPORTED).
+ * ------------------------------------------------------------------------- */
+size_t tsd_verify_attention_fp8_cache_workspace_bytes(const tsd_layout* layout);
+int tsd_verify_attention_fp8_cache(const tsd_layout* layout, const void* mask, const void* q,
+                                   int64_t q_stride_b, int64_t q_stride_row, int64_t q_stride_head,
+                                   const uint8_t* k_cache_e4m3, const uint8_t* v_cache_e4m3,
+                                   int64_t c_stride_b, int64_t c_stride_row, int64_t c_stride_head,
+                                   const float* k_scale, const float* v_scale, const void* k_draft,
+                                   const void* v_draft, int64_t d_stride_b, int64_t d_stride_row,
+                                   int64_t d_stride_head, void* out, int64_t o_stride_b,
+                                   int64_t o_stride_row, int64_t o_stride_head, float* lse,
+                                   float sm_scale, void* workspace, size_t workspace_bytes,
+                                   uint32_t flags, uint32_t* status, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
  * Stage 2 — confidence and candidates (Eq. 2: c = max softmax(logits);
  * Section 3.2: top-k candidates per position).  One streaming pass over the
  * logits.  Per row: conf = largest softmax probability; topk_idx = the k first

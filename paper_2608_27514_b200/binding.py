@@ -28,7 +28,7 @@ EXPORTS = (
     "tsd_confidence_topk_static_capacity", "tsd_confidence_topk_static",
     "tsd_accept_trajectories", "tsd_build_draft_tree",
     "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees", "tsd_accept_relaxed",
-    "tsd_commit_accepted",
+    "tsd_commit_accepted", "tsd_verify_attention_fp8_cache_workspace_bytes", "tsd_verify_attention_fp8_cache",
 )
 
 
@@ -92,6 +92,11 @@ def lib():
                                           _i64, _i64, _vp, _f32, _i32, _i32] + [_vp] * 10)
         L.tsd_commit_accepted.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _vp, _vp,
                                           _vp, _vp, _vp, _vp, _vp]
+        L.tsd_verify_attention_fp8_cache_workspace_bytes.restype = _sz
+        L.tsd_verify_attention_fp8_cache_workspace_bytes.argtypes = [ctypes.POINTER(tsd_layout)]
+        L.tsd_verify_attention_fp8_cache.argtypes = (
+            [ctypes.POINTER(tsd_layout), _vp] + [_vp, _i64, _i64, _i64] + [_vp, _vp, _i64, _i64, _i64, _vp, _vp]
+            + [_vp, _vp, _i64, _i64, _i64] + [_vp, _i64, _i64, _i64] + [_vp, _f32, _vp, _sz, _u32, _vp, _vp])
         _lib = L
     return _lib
 
@@ -300,3 +305,21 @@ def tsd_commit_accepted(parent, state, accepted_node, unmask_flag, unmask_tok, m
         int(mask_id), _ptr(tokens), 0 if tokens is None else tokens.stride(0), _ptr(block_start), _ptr(root_out),
         _ptr(fill_step), _ptr(step_base), _ptr(n_masked), _ptr(status), _stream(stream))
     _check(rc, "tsd_commit_accepted")
+
+
+def tsd_verify_attention_fp8_cache_workspace_bytes(layout):
+    return int(lib().tsd_verify_attention_fp8_cache_workspace_bytes(ctypes.byref(layout)))
+
+
+def tsd_verify_attention_fp8_cache(layout, mask, q, k_cache_e4m3, v_cache_e4m3, k_scale, v_scale, k_draft, v_draft,
+                                   out, workspace, lse=None, sm_scale=1.0, flags=0, status=None, stream=None):
+    """k/v_cache_e4m3: uint8 (or float8_e4m3fn) tensors [S, Nc, Hkv, d]; k/v_scale fp32 [S, Hkv] or None."""
+    assert v_cache_e4m3 is None or v_cache_e4m3.stride() == k_cache_e4m3.stride()
+    assert v_draft.stride() == k_draft.stride()
+    cs = _strides3(k_cache_e4m3) if k_cache_e4m3 is not None else (0, 0, layout.head_dim)
+    rc = lib().tsd_verify_attention_fp8_cache(
+        ctypes.byref(layout), _ptr(mask), _ptr(q), *_strides3(q), _ptr(k_cache_e4m3), _ptr(v_cache_e4m3), *cs,
+        _ptr(k_scale), _ptr(v_scale), _ptr(k_draft), _ptr(v_draft), *_strides3(k_draft), _ptr(out), *_strides3(out),
+        _ptr(lse), float(sm_scale), _ptr(workspace), workspace.numel() * workspace.element_size(), int(flags),
+        _ptr(status), _stream(stream))
+    _check(rc, "tsd_verify_attention_fp8_cache")
