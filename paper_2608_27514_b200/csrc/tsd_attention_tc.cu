@@ -618,16 +618,25 @@ static bool make_map(CUtensorMap* m, const void* ptr, int S, int rows, int H, in
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Per-device facts and one-time setup (a process may drive several GPUs).
+constexpr int kMaxDevices = 64;
+static int current_device() {
+  int dev = 0;
+  return cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices ? dev : -1;
+}
+
 static bool device_is_sm100() {
-  static int cached = -1;
-  if (cached < 0) {
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
-      return false;
-    cached = major == 10 ? 1 : 0;
+  static std::mutex mu;
+  static int cached[kMaxDevices];  // 0 = unknown, 1 = yes, 2 = no
+  const int dev = current_device();
+  if (dev < 0) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+    cached[dev] = major == 10 ? 1 : 2;
   }
-  return cached == 1;
+  return cached[dev] == 1;
 }
 
 bool attention_tc_supported(const AttnArgs& a) {
@@ -652,12 +661,19 @@ int launch_attention_tc(const AttnArgs& a) {
     mvc = mvd;
   }
   if (!ok) return launch_attention_simt(a);  // strides the tensor maps cannot express
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-  });
-  if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(attention_tc_kernel)");
+  {  // the dynamic shared memory limit is an attribute of the kernel on each device
+    static std::mutex mu;
+    static bool done[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return cuda_fail(cudaErrorInvalidDevice, "cudaGetDevice");
+    std::lock_guard<std::mutex> lock(mu);
+    if (!done[dev]) {
+      cudaError_t attr_err =
+          cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+      if (attr_err != cudaSuccess) return cuda_fail(attr_err, "cudaFuncSetAttribute(attention_tc_kernel)");
+      done[dev] = true;
+    }
+  }
   TcParams p;
   p.mask = a.mask;
   p.out = static_cast<__nv_bfloat16*>(a.out);
