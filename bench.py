@@ -452,7 +452,10 @@ def main():
     stages = dict(
         attention=dict(seconds=t_attn, bound=attn_bound, roofline_seconds=max(attn_flop_time, attn_byte_time),
                        frac=max(attn_flop_time, attn_byte_time) / t_attn,
-                       tflops=alg["attn_flops"] / t_attn / 1e12, gbs=alg["attn_bytes"] / t_attn / 1e9),
+                       tflops=alg["attn_flops"] / t_attn / 1e12, gbs=alg["attn_bytes"] / t_attn / 1e9,
+                       # the stage loop runs for a quarter of a second under the power cap: the fraction
+                       # of the sustained cuBLAS figure is given beside the (conservative) burst one
+                       frac_of_sustained_tensor_peak=alg["attn_flops"] / t_attn / 1e12 / pk["tflops_sustained"]),
         topk=dict(seconds=t_topk, bound="hbm", roofline_seconds=alg["topk_bytes"] / (pk["hbm_gbs"] * 1e9),
                   frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9),
         accept=dict(seconds=t_acc),
