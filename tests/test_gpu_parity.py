@@ -116,6 +116,34 @@ def test_attention_small_bf16_ragged_gqa(flags, R):
 
 
 @pytest.mark.parametrize("flags", PATHS)
+def test_attention_strided_views_of_packed_tensors(flags):
+    # Q / draft K / draft V as slices of one fused projection output, cached K / V as slices of one
+    # cache tensor, the output as a view into a wider buffer: same bits as the contiguous call
+    cfg = W.small(W.CONFIGS["cfg2"], S=2, B=5, R=32, Nc=200, Hq=4, Hkv=2)
+    attn = W.attention_inputs(cfg, DEV)
+    step, _ = _run_attention(cfg, attn, flags)
+    ref_out, ref_lse = step.out.clone(), step.attn_lse.clone()
+    qkv = torch.empty((cfg.S, cfg.N, cfg.Hq + 2 * cfg.Hkv, cfg.d), dtype=attn["q"].dtype, device=DEV)
+    qkv[:, :, :cfg.Hq] = attn["q"]
+    qkv[:, :, cfg.Hq:cfg.Hq + cfg.Hkv] = attn["k_draft"]
+    qkv[:, :, cfg.Hq + cfg.Hkv:] = attn["v_draft"]
+    cache = torch.empty((cfg.S, cfg.Nc, 2 * cfg.Hkv, cfg.d), dtype=attn["q"].dtype, device=DEV)
+    cache[:, :, :cfg.Hkv] = attn["k_cache"]
+    cache[:, :, cfg.Hkv:] = attn["v_cache"]
+    wide = torch.full((cfg.S, cfg.N + 3, cfg.Hq + 1, cfg.d), 9.0, dtype=attn["q"].dtype, device=DEV)
+    out = wide[:, 1:cfg.N + 1, :cfg.Hq]
+    step2 = VerifyStep.for_config(cfg, DEV)
+    step2.build_mask()
+    step2.attention(qkv[:, :, :cfg.Hq], cache[:, :, :cfg.Hkv], cache[:, :, cfg.Hkv:],
+                    qkv[:, :, cfg.Hq:cfg.Hq + cfg.Hkv], qkv[:, :, cfg.Hq + cfg.Hkv:], attn["sm_scale"], flags, out=out)
+    torch.cuda.synchronize()
+    step2.check_status()
+    assert torch.equal(out, ref_out) and torch.equal(step2.attn_lse, ref_lse)
+    # nothing outside the view was touched
+    assert (wide[:, 0] == 9.0).all() and (wide[:, cfg.N + 1:] == 9.0).all() and (wide[:, :, cfg.Hq] == 9.0).all()
+
+
+@pytest.mark.parametrize("flags", PATHS)
 def test_attention_custom_visibility(flags):
     # asymmetric visibility as in the inter-block variant (Section 3.4): drafts read the root
     cfg = W.small(W.CONFIGS["cfg2"], S=2, B=7, R=32, Nc=128, Hq=2, Hkv=2)
