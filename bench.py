@@ -208,6 +208,7 @@ def main():
     ap.add_argument("--impl", default="tsd", choices=["tsd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graph replay")
+    ap.add_argument("--graph-per-step", action="store_true", help="one graph launch per step instead of one per round of input copies")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tsd" else args.warmup
 
@@ -252,7 +253,8 @@ def main():
         step, attn, vi = sets[i % n_copies]
         step.run(attn, vi["logits"], vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
 
-    graphs = None
+    graphs = round_graph = None
+    round_len = n_copies if n_copies > 1 else 4  # steps per round graph (a multiple of the input copies)
     use_graph = not args.no_graph
     if use_graph:
         # one captured step per input copy; the library calls only enqueue work, so they capture as is
@@ -269,26 +271,43 @@ def main():
             with torch.cuda.graph(g):
                 run_step(i)
             graphs.append(g)
+        # and one graph holding a round of consecutive steps (one per input copy), the way a decode
+        # loop is captured: replaying it costs one graph launch per round instead of one per step
+        round_graph = None
+        if not args.graph_per_step:
+            round_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(round_graph):
+                for i in range(round_len):
+                    run_step(i)
 
-    def do_step(i):
-        if graphs is not None:
-            graphs[i % n_copies].replay()
-        else:
-            run_step(i)
+    def do_steps(first, count):
+        """Steps first .. first + count - 1, each on input copy (step index % n_copies)."""
+        i, end = first, first + count
+        while i < end:
+            if graphs is None:
+                run_step(i)
+                i += 1
+            elif round_graph is not None and i % round_len == 0 and i + round_len <= end:
+                round_graph.replay()
+                i += round_len
+            else:
+                graphs[i % n_copies].replay()
+                i += 1
 
     def barrier():
         replicas.barrier()
         torch.cuda.synchronize()
 
     # ---------------- timed region A: K whole steps, inputs resident in HBM
-    for i in range(args.warmup):
-        do_step(i)
+    first = -(-args.warmup // round_len) * round_len  # the timed steps start on a round boundary
+    do_steps(first - args.warmup, args.warmup)
+    if round_graph is not None:
+        round_graph.replay()   # the round graph itself warm (not counted)
     sampler = ClockSampler(local_rank)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(args.steps):
-        do_step(args.warmup + i)
+    do_steps(first, args.steps)
     e1.record(stream)
     barrier()
     elapsed_ms = e0.elapsed_time(e1)
@@ -509,7 +528,9 @@ def main():
                     l2_hygiene=("inputs larger than L2" if n_copies == 1 else
                                 "rotating %d input copies (%.0f MB total, L2 is 126 MB)"
                                 % (n_copies, n_copies * in_bytes / 1e6)),
-                    launch="cuda graph replay" if graphs is not None else "plain launches"),
+                    launch=("plain launches" if graphs is None else
+                            "cuda graph replay, one graph per step" if round_graph is None else
+                            "cuda graph replay, one graph per round of %d steps" % round_len)),
         clocks=clocks,
         e2e=dict(value=world * cfg.rows / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(h2d),
                  d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms),
