@@ -24,7 +24,8 @@ namespace tsd {
 constexpr int kMaxBranches = 256;
 constexpr int kMaxRows = 128;
 constexpr int kRowWords = kMaxRows / 32;
-constexpr int kAcceptThreads = 256;
+constexpr int kAcceptThreads = 256;      // a warp per node up to 8 nodes ...
+constexpr int kAcceptMaxThreads = 1024;  // ... and up to 32 warps for larger trees (nodes are taken in turn)
 
 struct RelaxedArgs {
   int topk_m;           // candidates per row that count for TSD_ACCEPT_TOPK
@@ -35,7 +36,7 @@ struct RelaxedArgs {
   float* draft_prob;    // [batch, B, R] out, nullable
 };
 
-__global__ void __launch_bounds__(kAcceptThreads)
+__global__ void __launch_bounds__(kAcceptMaxThreads)
 accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
               int mask_id, const float* __restrict__ conf, const int32_t* __restrict__ top1,
               int top1_stride, float tau, int rule, int search, uint8_t* __restrict__ edge_valid,
@@ -238,7 +239,10 @@ static int accept_launch(int32_t batch, int32_t n_branches, int32_t n_cur, int32
       !accepted_len || !n_new_tokens || !unmask_flag || !unmask_tok)
     return TSD_ERR_INVALID_ARG;
   const dim3 grid(batch, n_cur < n_branches ? 2 : 1);
-  tsd::accept_kernel<<<grid, tsd::kAcceptThreads, 0, stream>>>(
+  const int tree_max = n_cur > n_branches - n_cur ? n_cur : n_branches - n_cur;
+  const int threads = tree_max * 32 < tsd::kAcceptThreads ? tsd::kAcceptThreads
+                      : (tree_max * 32 > tsd::kAcceptMaxThreads ? tsd::kAcceptMaxThreads : tree_max * 32);
+  tsd::accept_kernel<<<grid, threads, 0, stream>>>(
       n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
       search, edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
       unmask_tok, status, x);
