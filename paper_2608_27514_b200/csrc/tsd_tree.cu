@@ -53,6 +53,10 @@ __device__ __forceinline__ Cand warp_best(Cand c) {
   return c;
 }
 
+// RPL = rows per lane (R <= 32 * RPL), KK = candidates per row held in registers (k <= KK): the
+// selection loops are unrolled over RPL x KK, so the common block of 32 rows with k <= 4 runs a
+// tenth of the instructions of the largest case (a single warp is bound by instruction latency).
+template <int RPL, int KK>
 __global__ void __launch_bounds__(32)
 build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restrict__ prev_state,
                         const int32_t* __restrict__ accepted_node, const uint8_t* __restrict__ unmask_flag,
@@ -65,7 +69,7 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
   __shared__ int s_front[kTreeMaxWidth];
   __shared__ int s_cpar[kTreeMaxWidth], s_crow[kTreeMaxWidth], s_crank[kTreeMaxWidth];
   __shared__ float s_cp[kTreeMaxWidth];
-  __shared__ uint32_t s_mask[256][kTreeRowsPerLane];  // per node: which rows are still masked
+  __shared__ uint32_t s_mask[256][RPL];  // per node: which rows are still masked
   const int s = blockIdx.x, lane = threadIdx.x;
   int acc = accepted_node ? accepted_node[s] : 0;
   if (acc < 0 || acc >= prev_branches) {  // inconsistent device data: report, fall back to node 0
@@ -81,9 +85,9 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
   if (enable && !enable[s]) D = 0;
 
   // next root = accepted state + its unmask set; every node slot starts as a copy of it
-  bool root_masked[kTreeRowsPerLane];
+  bool root_masked[RPL];
 #pragma unroll
-  for (int i = 0; i < kTreeRowsPerLane; ++i) {
+  for (int i = 0; i < RPL; ++i) {
     const int r = lane + 32 * i;
     root_masked[i] = false;
     if (r < R) {
@@ -99,12 +103,12 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
   }
   // the pool lives in registers (this lane's rows x k) and the nodes' masked-row sets in shared
   // memory, so the selection rounds below touch no global memory
-  float pool[kTreeRowsPerLane][kTreeMaxK];
+  float pool[RPL][KK];
 #pragma unroll
-  for (int i = 0; i < kTreeRowsPerLane; ++i) {
+  for (int i = 0; i < RPL; ++i) {
     const int r = lane + 32 * i;
 #pragma unroll
-    for (int j = 0; j < kTreeMaxK; ++j) pool[i][j] = (r < R && j < k) ? prb[(size_t)r * k + j] : -1.f;
+    for (int j = 0; j < KK; ++j) pool[i][j] = (r < R && j < k) ? prb[(size_t)r * k + j] : -1.f;
     const uint32_t word = __ballot_sync(0xffffffffu, root_masked[i]);
     if (lane == 0) s_mask[0][i] = word;
   }
@@ -120,12 +124,12 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
       for (int t = 0; t < k; ++t) {
         Cand best = {0.f, -1, 0};
 #pragma unroll
-        for (int i = 0; i < kTreeRowsPerLane; ++i) {
+        for (int i = 0; i < RPL; ++i) {
           const int r = lane + 32 * i;
           if (r < R && root_masked[i]) {
 #pragma unroll
-            for (int j = 0; j < kTreeMaxK; ++j) {
-              if (j >= k || ((used >> (i * kTreeMaxK + j)) & 1u)) continue;
+            for (int j = 0; j < KK; ++j) {
+              if (j >= k || ((used >> (i * KK + j)) & 1u)) continue;
               const Cand c = {pool[i][j], r, j};
               if (cand_before(c, best)) best = c;
             }
@@ -133,7 +137,7 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
         }
         const Cand win = warp_best(best);
         if (win.row < 0) break;  // pool exhausted (uniform: every lane sees the same winner)
-        if ((win.row & 31) == lane) used |= 1u << ((win.row >> 5) * kTreeMaxK + win.rank);
+        if ((win.row & 31) == lane) used |= 1u << ((win.row >> 5) * KK + win.rank);
         if (lane == 0) { s_cpar[n_child] = 0; s_crow[n_child] = win.row; s_crank[n_child] = win.rank; s_cp[n_child] = win.p; }
         ++n_child;
       }
@@ -142,11 +146,11 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
         const int node = s_front[f];
         Cand best = {0.f, -1, 0};
 #pragma unroll
-        for (int i = 0; i < kTreeRowsPerLane; ++i) {
+        for (int i = 0; i < RPL; ++i) {
           const int r = lane + 32 * i;
           if (r < R && ((s_mask[node][i] >> lane) & 1u)) {
 #pragma unroll
-            for (int j = 0; j < kTreeMaxK; ++j) {
+            for (int j = 0; j < KK; ++j) {
               if (j >= k) continue;
               const Cand c = {pool[i][j], r, j};
               if (cand_before(c, best)) best = c;
@@ -191,7 +195,7 @@ build_draft_tree_kernel(int prev_branches, int R, int k, const int32_t* __restri
       const int crow = __shfl_sync(0xffffffffu, my_row, owner);
       const int ctok = __shfl_sync(0xffffffffu, my_tok, owner);
 #pragma unroll
-      for (int i = 0; i < kTreeRowsPerLane; ++i) {
+      for (int i = 0; i < RPL; ++i) {
         const int r = lane + 32 * i;
         if (r < R) st[(size_t)(n + q) * R + r] = r == crow ? ctok : st[(size_t)cpar * R + r];
         if (lane == 0) s_mask[n + q][i] = s_mask[cpar][i] & ~((crow >> 5) == i ? (1u << (crow & 31)) : 0u);
@@ -222,10 +226,15 @@ extern "C" int tsd_build_draft_tree(int32_t batch, int32_t prev_branches, int32_
   if (batch == 0) return TSD_OK;
   if (!prev_state || !topk_idx || !topk_prob || !parent || !state || !node_prob || !n_nodes)
     return TSD_ERR_INVALID_ARG;
-  tsd::build_draft_tree_kernel<<<batch, 32, 0, stream>>>(
-      prev_branches, rows_per_branch, k, prev_state, accepted_node, unmask_flag, unmask_tok, mask_id, topk_idx,
-      topk_prob, width, depth, max_nodes, out_stride, node_base, enable, parent, state, node_prob, n_nodes,
-      status);
+  auto launch = [&](auto kernel) {
+    kernel<<<batch, 32, 0, stream>>>(prev_branches, rows_per_branch, k, prev_state, accepted_node, unmask_flag,
+                                     unmask_tok, mask_id, topk_idx, topk_prob, width, depth, max_nodes, out_stride,
+                                     node_base, enable, parent, state, node_prob, n_nodes, status);
+  };
+  const int rpl = (rows_per_branch + 31) / 32;
+  if (rpl == 1 && k <= 4) launch(tsd::build_draft_tree_kernel<1, 4>);
+  else if (rpl <= 2 && k <= 4) launch(tsd::build_draft_tree_kernel<2, 4>);
+  else launch(tsd::build_draft_tree_kernel<tsd::kTreeRowsPerLane, tsd::kTreeMaxK>);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return tsd::cuda_fail(e, "build_draft_tree_kernel");
   return TSD_OK;
