@@ -36,6 +36,8 @@ struct RelaxedArgs {
   float* draft_prob;    // [batch, B, R] out, nullable
 };
 
+// WORDS = 32-row words per node that the unrolled loops cover (R <= 32 * WORDS).
+template <int WORDS>
 __global__ void __launch_bounds__(kAcceptMaxThreads)
 accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
               int mask_id, const float* __restrict__ conf, const int32_t* __restrict__ top1,
@@ -60,15 +62,15 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   const int32_t* st = state + ((size_t)s * B_all + lo) * R;
   const float* cf = conf + ((size_t)s * B_all + lo) * R;
   const int32_t* t1 = top1 + ((size_t)s * B_all + lo) * R * top1_stride;
-  const int words = (R + 31) / 32;
+  const int words = min((R + 31) / 32, WORDS);
 
   // decode rule U(p) for every node
   for (int p = warp; p < B; p += n_warps) {
-    uint32_t hi[kRowWords], any_hi = 0, any_masked = 0;
+    uint32_t hi[WORDS], any_hi = 0, any_masked = 0;
     float best = -CUDART_INF_F;
     int best_r = INT_MAX;
 #pragma unroll
-    for (int w = 0; w < kRowWords; ++w) {
+    for (int w = 0; w < WORDS; ++w) {
       hi[w] = 0;
       if (w < words) {
         const int r = w * 32 + lane;
@@ -95,11 +97,11 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
         if (take) { best = ov; best_r = orow; }
       }
 #pragma unroll
-      for (int w = 0; w < kRowWords; ++w) hi[w] = (best_r >> 5) == w ? (1u << (best_r & 31)) : 0u;
+      for (int w = 0; w < WORDS; ++w) hi[w] = (best_r >> 5) == w ? (1u << (best_r & 31)) : 0u;
     }
     if (lane == 0) {
 #pragma unroll
-      for (int w = 0; w < kRowWords; ++w) s_u[p][w] = hi[w];
+      for (int w = 0; w < WORDS; ++w) s_u[p][w] = hi[w];
       int par = -1;
       if (p > 0) {
         const int raw = parent[(size_t)s * B_all + lo + p];  // forest index
@@ -242,7 +244,9 @@ static int accept_launch(int32_t batch, int32_t n_branches, int32_t n_cur, int32
   const int tree_max = n_cur > n_branches - n_cur ? n_cur : n_branches - n_cur;
   const int threads = tree_max * 32 < tsd::kAcceptThreads ? tsd::kAcceptThreads
                       : (tree_max * 32 > tsd::kAcceptMaxThreads ? tsd::kAcceptMaxThreads : tree_max * 32);
-  tsd::accept_kernel<<<grid, threads, 0, stream>>>(
+  auto kernel = rows_per_branch <= 32 ? tsd::accept_kernel<1>
+                : rows_per_branch <= 64 ? tsd::accept_kernel<2> : tsd::accept_kernel<tsd::kRowWords>;
+  kernel<<<grid, threads, 0, stream>>>(
       n_branches, n_cur, rows_per_branch, parent, state, mask_id, conf, top1_idx, top1_stride, tau, rule,
       search, edge_valid, prefix_len, accepted_node, accepted_len, n_new_tokens, unmask_flag,
       unmask_tok, status, x);
