@@ -29,14 +29,14 @@ ROTATE_BYTES = 640 * 1024 * 1024  # rotate through input copies at least this la
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (kernel -> workload -> bytes); None where no capture exists.
 NCU_TRAFFIC = {
-    # cfg2: measured on this workload (profiles/bench_cfg2_launch_list.md).  Others: the 2048-row
-    # capture (523.9 MB, profiles/confidence_topk_kernel_2048rows_v126464.md) scaled by logit bytes,
+    # cfg2: measured on this workload (the launch-list capture under profiles/).  Others: the 2048-row
+    # capture (523.9 MB, the top-k capture under profiles/) scaled by logit bytes,
     # traffic being proportional to them.
     "confidence_topk": {"cfg2": 64.8e6, "cfg3": 523.9e6 * 1024 / 2048, "cfg4": 523.9e6 * 16384 / 2048,
                         "cfg5": 523.9e6 * 16384 / 2048 * 152064 / 126464},
     # cfg2: measured on this workload; cfg4: the 4-sequence capture (223.4 MB) x 4; cfg5: an earlier
     # 1-sequence capture (49.6 MB, part of the output still in L2) x 4
-    # (profiles/attention_tc_kernel_cfg4_4seq.md).
+    # (the attention capture under profiles/).
     "verify_attention": {"cfg2": 18.4e6, "cfg4": 223.4e6 * 4, "cfg5": 49.6e6 * 4},
 }
 
