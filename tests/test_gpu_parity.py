@@ -115,6 +115,29 @@ def test_attention_small_bf16_ragged_gqa(flags, R):
     _check_attention(cfg, attn, flags, cache_lens=lens)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_attention_random_shapes_masks_and_cache_lengths(seed):
+    # shapes, visibility bitsets and cache lengths drawn at random: partial query tiles, empty and
+    # ragged caches, grouped heads, branches that read several others
+    rng = np.random.default_rng(100 + seed)
+    R = int(rng.choice([32, 64, 128]))
+    Bn = int(rng.integers(1, 21 if R == 32 else 9))
+    Hkv = int(rng.choice([1, 2]))
+    Hq = Hkv * int(rng.choice([1, 2, 3]))
+    cfg = W.small(W.CONFIGS["cfg2"], S=int(rng.integers(1, 4)), B=Bn, R=R, Nc=int(rng.choice([0, 1, 63, 64, 65, 200, 333])),
+                  Hq=Hq, Hkv=Hkv)
+    vis = np.zeros((cfg.S, Bn, 1), dtype=np.int64)
+    for s_ in range(cfg.S):
+        for b in range(Bn):
+            if rng.random() < 0.4:
+                vis[s_, b, 0] = int(rng.integers(0, 1 << Bn))
+    cache_lens = None
+    if cfg.Nc:
+        cache_lens = torch.from_numpy(rng.integers(0, cfg.Nc + 1, cfg.S).astype(np.int32)).to(DEV)
+    flags = B.TSD_ATTN_FORCE_SIMT if seed % 4 == 3 else 0
+    _check_attention(cfg, W.attention_inputs(cfg, DEV), flags, vis=torch.from_numpy(vis).to(DEV), cache_lens=cache_lens)
+
+
 @pytest.mark.parametrize("flags", PATHS)
 def test_attention_strided_views_of_packed_tensors(flags):
     # Q / draft K / draft V as slices of one fused projection output, cached K / V as slices of one
