@@ -275,6 +275,28 @@ def test_topk_ragged_vocab_and_heavy_ties(dtype, k):
         _check_topk(buf[:, :V], min(k, V))
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_topk_random_rows_vocab_k_and_dtype(seed):
+    # sizes drawn at random: one value per row up to a wide vocabulary, one row up to several waves of
+    # blocks, segmented and whole rows, ragged tails, a sharp peak in some rows, -inf in others
+    rng = np.random.default_rng(500 + seed)
+    V = int(rng.choice([1, 2, 7, 8, 9, 31, 257, 1000, 4099, 20000, 70001]))
+    n = int(rng.choice([1, 2, 5, 40, 147, 149, 300, 700]))
+    if n * V > 30_000_000:
+        n = max(1, 30_000_000 // V)
+    k = int(min(rng.integers(1, 9), V))
+    dtype = torch.float32 if seed % 2 else torch.bfloat16
+    pitch = (V + 7) // 8 * 8
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    buf = (torch.randn((n, pitch), generator=g, device=DEV) * float(rng.choice([0.5, 3.0, 10.0]))).to(dtype)
+    x = buf[:, :V]
+    rows = torch.arange(n, device=DEV)
+    x[rows[::3], torch.randint(0, V, (len(rows[::3]),), generator=g, device=DEV)] += 12.0      # sharp peaks
+    if V > 4:
+        x[rows[1::4], :2] = float("-inf")
+    _check_topk(x, k)
+
+
 def test_topk_minus_inf_and_split_rows():
     V = 126464
     g = torch.Generator(device=DEV).manual_seed(5)
