@@ -228,8 +228,8 @@ int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32
  *     (cudaGetSymbolAddress, with that device current).  Make that first call
  *     before any stream capture begins.
  *   - All calls on a device share the one array, and it keeps whatever the
- *     previous call left: each call re-zeroes the ticket words it uses (on
- *     `stream`, ahead of its kernel) and overwrites the partial slots it reads.
+ *     previous call left: a completed call leaves every ticket word it used
+ *     idle again and the next call overwrites the partial slots it reads.
  *     Two calls that overlap on the GPU (different streams, no ordering) would
  *     race on it: order them on one stream or with events.
  * Arguments as for tsd_confidence_topk, minus the workspace.

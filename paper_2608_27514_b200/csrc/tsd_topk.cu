@@ -7,15 +7,16 @@
 //      takes the packed maximum of its 32 values, rebases its running sum to the new maximum with
 //      one multiply, adds 2^(x*log2e - e) for every value (one FFMA + one ex2 each), and stores the
 //      batch maximum in shared memory.
-//   2. bound: the k-th largest of the 256 per-thread maxima (warp shuffles, then across warps).
-//      At least k values of the row are >= it, so it is a valid lower bound of the k-th best.
-//   3. collect: each thread re-reads only those of its batches whose maximum reaches the bound
-//      (a handful per row, served by L2) and inserts the values >= bound into a sorted k-entry
-//      list in registers; lists are merged by warp shuffles (k rounds of an arg-best reduction),
-//      then across the warps of the block through shared memory.
+//   2. bound: the k-th largest of the warps' maxima (one shuffle reduction per warp, then every
+//      thread selects among the 8 or 16 values in registers).  At least k values of the row are
+//      >= it, so it is a valid lower bound of the k-th best.
+//   3. collect: each warp re-reads only those of its batches whose maximum reaches the bound
+//      (a handful per row, served by L2); the values >= bound go into a small pool in shared
+//      memory, from which one warp picks the k best by counting ranks (no sort, no shuffles).
+//      A pool that would overflow (heavy ties) falls back to merging per-lane lists by shuffles.
 // With few rows a row is split into segments handled by different blocks; the last block to finish
-// a row (a ticket counter in the workspace, no spinning) merges the segment partials in segment
-// order, so the result does not depend on arrival order.
+// a row (a ticket word in the workspace, no spinning, no clearing between calls) merges the
+// segment partials in segment order, so the result does not depend on arrival order.
 //
 // Ordering is (logit descending, index ascending) on the raw input values (bf16 and fp32 both
 // widen to fp32 exactly), so indices are uniquely defined.
@@ -30,6 +31,8 @@ namespace tsd {
 constexpr int kTopkUnroll = 4;            // chunks per thread per batch
 constexpr int kTopkSegChunks = 32768;     // chunks per segment at most (batch maxima: 32 KB of smem)
 constexpr int kMaxSegments = 32;
+constexpr int kPoolCap = 64;              // candidate pool of a block (entries)
+constexpr unsigned kTicketTag = 0x7FC3A9u;  // upper 24 bits of a ticket word that is in use
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ bool key_before(float va, int ia, float vb, int ib) {
@@ -154,21 +157,6 @@ __device__ __forceinline__ void warp_merge(Acc<K>& a) {
   a.e = a.seen ? E : 0.f;
 }
 
-// k-th largest of the values held one per lane (K rounds; equal values leave together, which can
-// only lower the result, so it stays a valid lower bound).  Every lane gets the result.
-template <int K>
-__device__ __forceinline__ void warp_top_values(float x, float (&top)[K]) {
-  const unsigned full = 0xffffffffu;
-#pragma unroll
-  for (int r = 0; r < K; ++r) {
-    float b = x;
-#pragma unroll
-    for (int off = 16; off; off >>= 1) b = fmaxf(b, __shfl_xor_sync(full, b, off));
-    top[r] = b;
-    if (x == b) x = -CUDART_INF_F;
-  }
-}
-
 template <int K>
 struct Partial {  // one segment's result, as stored in the workspace
   float e, s;     // e = -inf when nothing finite was seen
@@ -176,8 +164,9 @@ struct Partial {  // one segment's result, as stored in the workspace
   int i[K];
 };
 
+// Every lane of the warp holds the merged result; lane j writes candidate j.
 template <int K>
-__device__ __forceinline__ void finalize(const Acc<K>& a, int k, int64_t row, float* conf,
+__device__ __forceinline__ void finalize(const Acc<K>& a, int k, int64_t row, int lane, float* conf,
                                          int32_t* topk_idx, float* topk_prob, float* lse) {
   // a.s = sum 2^(x*log2e - e) with e = fl(M*log2e): the FMA residual d = M*log2e - e is exact
   const float M = a.v[0];
@@ -186,14 +175,28 @@ __device__ __forceinline__ void finalize(const Acc<K>& a, int k, int64_t row, fl
   const float inv = 1.f / Z;
 #pragma unroll
   for (int j = 0; j < K; ++j) {
-    if (j < k) {
+    if (j == lane && j < k) {
       const float p = expf(a.v[j] - M) * inv;
       topk_idx[row * k + j] = a.i[j];
       topk_prob[row * k + j] = p;
       if (j == 0) conf[row] = p;
     }
   }
-  if (lse) lse[row] = M + logf(Z);
+  if (lse && lane == 0) lse[row] = M + logf(Z);
+}
+
+// One arrival on a row's ticket word; true for the last of n_seg arrivals, which also returns the
+// word to idle.  A word in use carries kTicketTag in its upper 24 bits and the number of arrivals
+// so far in the lower 8; any other content counts as idle, so the workspace needs no clearing.
+__device__ __forceinline__ bool ticket_arrive(unsigned* t, int n_seg) {
+  unsigned old = *reinterpret_cast<volatile unsigned*>(t), assumed, cnt;
+  do {
+    assumed = old;
+    cnt = (assumed >> 8) == kTicketTag ? (assumed & 0xffu) : 0u;
+    const unsigned next = (cnt + 1 == (unsigned)n_seg) ? 0u : ((kTicketTag << 8) | (cnt + 1));
+    old = atomicCAS(t, assumed, next);
+  } while (old != assumed);
+  return cnt + 1 == (unsigned)n_seg;
 }
 
 template <typename T>
@@ -262,23 +265,29 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
                        int chunks_per_seg, float* __restrict__ conf, int32_t* __restrict__ topk_idx,
                        float* __restrict__ topk_prob, float* __restrict__ lse,
                        Partial<K>* __restrict__ partials, unsigned* __restrict__ tickets, int prefetch) {
-  constexpr int E = Unpack<T>::kElems;
+  constexpr int E_ = Unpack<T>::kElems;
   constexpr int kTopkThreads = THREADS, kTopkWarps = THREADS / 32;
   constexpr int kTopkBatch = THREADS * kTopkUnroll;        // chunks per block per batch
   constexpr int kTopkMaxIter = kTopkSegChunks / kTopkBatch;  // batches per segment
   __shared__ float s_bmax[kTopkMaxIter][kTopkThreads];  // per-thread batch maxima
-  __shared__ float s_top[kTopkWarps][K];
-  __shared__ Partial<K> s_part[kTopkWarps];
+  __shared__ __align__(16) float s_wmax[kTopkWarps];  // per-warp maxima
+  __shared__ float s_wsum[kTopkWarps];                // per-warp sums on the block's exponent base
+  __shared__ float s_pool_v[kPoolCap];                // candidates found by the collect phase
+  __shared__ int s_pool_i[kPoolCap];
+  __shared__ int s_cnt;
+  __shared__ float s_res_v[K];
+  __shared__ int s_res_i[K];
+  __shared__ Partial<K> s_part[kTopkWarps];           // shuffle-merge path only
   const int64_t row = blockIdx.x / n_seg;
   const int seg = blockIdx.x % n_seg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const T* rowp = logits + row * row_stride;
   const uint4* rowv = reinterpret_cast<const uint4*>(rowp);
-  const int chunks_total = vocab / E;
+  const int chunks_total = vocab / E_;
   const int c0 = seg * chunks_per_seg;
   const int c1 = min(c0 + chunks_per_seg, chunks_total);
   const int n_iter = (c1 - c0 + kTopkBatch - 1) / kTopkBatch;  // <= kTopkMaxIter (host-enforced)
-  const bool has_tail = seg == n_seg - 1 && tid == 0 && chunks_total * E < vocab;
+  const bool has_tail = seg == n_seg - 1 && tid == 0 && chunks_total * E_ < vocab;
 
   // ---- phase 1: stream.  Two register buffers: the loads of batch it+1 are in flight while
   // batch it is processed, so a block overlaps memory latency with its own arithmetic.
@@ -330,67 +339,75 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   }
   float tail_max = -CUDART_INF_F;
   if (has_tail) {  // ragged tail of a vocabulary that is not a multiple of the chunk size
-    for (int x = chunks_total * E; x < vocab; ++x) tail_max = fmaxf(tail_max, to_float(rowp[x]));
+    for (int x = chunks_total * E_; x < vocab; ++x) tail_max = fmaxf(tail_max, to_float(rowp[x]));
     const float m_new = fmaxf(m, tail_max);
     const float e_new = (m_new == -CUDART_INF_F) ? 0.f : m_new * kLog2e;
     s *= (m == -CUDART_INF_F) ? 0.f : ex2_approx(e - e_new);
     m = m_new;
     e = e_new;
-    for (int x = chunks_total * E; x < vocab; ++x) s += ex2_approx(fmaf(to_float(rowp[x]), kLog2e, -e));
+    for (int x = chunks_total * E_; x < vocab; ++x) s += ex2_approx(fmaf(to_float(rowp[x]), kLog2e, -e));
   }
 
-  // ---- phase 2: bound = k-th largest per-thread maximum of the block
-  float top[K];
-  warp_top_values<K>(m, top);
-  if (lane == 0) {
+  // ---- phase 2: bound = k-th largest of the warps' maxima.  Each of the k best warps holds a
+  // value equal to its maximum, so at least k values of the piece reach the bound.  One shuffle
+  // reduction per warp; after the block-wide barrier every thread picks the k-th largest of the
+  // WARPS values in registers (no further shuffles or barriers).
+  if (tid == 0) s_cnt = 0;
+  {
+    float wm = m;
 #pragma unroll
-    for (int j = 0; j < K; ++j) s_top[warp][j] = top[j];
+    for (int off = 16; off; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+    if (lane == 0) s_wmax[warp] = wm;
   }
   __syncthreads();
+  float M = -CUDART_INF_F, bound = -CUDART_INF_F;
   {
-    // every warp redoes the small cross-warp step: the lanes hold the WARPS x K warp values
-    constexpr int NV = (kTopkWarps * K + 31) / 32;
-    float cv[NV];
+    float wv[kTopkWarps];
 #pragma unroll
-    for (int q = 0; q < NV; ++q) {
-      const int idx = lane + 32 * q;
-      cv[q] = idx < kTopkWarps * K ? s_top[idx / K][idx % K] : -CUDART_INF_F;
+    for (int q = 0; q < kTopkWarps / 4; ++q) {
+      const float4 f = reinterpret_cast<const float4*>(s_wmax)[q];
+      wv[4 * q] = f.x; wv[4 * q + 1] = f.y; wv[4 * q + 2] = f.z; wv[4 * q + 3] = f.w;
     }
-    float bound = -CUDART_INF_F;
 #pragma unroll
     for (int r = 0; r < K; ++r) {
-      float x = cv[0];
+      float x = wv[0];
 #pragma unroll
-      for (int q = 1; q < NV; ++q) x = fmaxf(x, cv[q]);
-#pragma unroll
-      for (int off = 16; off; off >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, off));
+      for (int q = 1; q < kTopkWarps; ++q) x = fmaxf(x, wv[q]);
+      if (r == 0) M = x;
       bound = x;
+      bool gone = false;  // one instance leaves per round: the k-th largest counts multiplicity
 #pragma unroll
-      for (int q = 0; q < NV; ++q)
-        if (cv[q] == x) cv[q] = -CUDART_INF_F;
+      for (int q = 0; q < kTopkWarps; ++q) {
+        const bool hit = !gone && wv[q] == x;
+        wv[q] = hit ? -CUDART_INF_F : wv[q];
+        gone = gone || hit;
+      }
     }
-    top[0] = bound;
   }
-  const float bound = top[0];
+  // the block's sum on the block's exponent base; the per-warp sums meet after the next barrier
+  const float E = (M == -CUDART_INF_F) ? 0.f : M * kLog2e;
+  {
+    float sr = (m == -CUDART_INF_F) ? 0.f : s * ex2_approx(e - E);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) sr += __shfl_xor_sync(0xffffffffu, sr, off);
+    if (lane == 0) s_wsum[warp] = sr;
+  }
 
   // ---- phase 3: collect the values >= bound from the few batches that hold one
   Acc<K> a;
   a.init();
-  a.seen = m != -CUDART_INF_F;
-  a.e = e;
-  a.s = s;
   // The whole block waits for its slowest warp here, so a hit batch (32 values for bf16, 16 for
   // fp32) is examined by the warp together: lane l re-reads value l of the batch (an L2 hit) and
-  // offers it to its own list; warp_merge combines the lanes' lists afterwards.
+  // offers it to its own list.
   for (int it = 0; it < n_iter; ++it) {
     unsigned hits = __ballot_sync(0xffffffffu, s_bmax[it][tid] >= bound);
     while (hits) {
       const int src = __ffs(hits) - 1;
       hits &= hits - 1;
-      if (lane < kTopkUnroll * E) {
-        const int c = c0 + it * kTopkBatch + (warp * 32 + src) + (lane / E) * kTopkThreads;
+      if (lane < kTopkUnroll * E_) {
+        const int c = c0 + it * kTopkBatch + (warp * 32 + src) + (lane / E_) * kTopkThreads;
         if (c < c1) {
-          const int xi = c * E + lane % E;
+          const int xi = c * E_ + lane % E_;
           const float x = to_float(rowp[xi]);
           if (x >= bound) a.offer(x, xi);
         }
@@ -398,36 +415,84 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     }
   }
   if (has_tail && tail_max >= bound) {
-    for (int x = chunks_total * E; x < vocab; ++x) {
+    for (int x = chunks_total * E_; x < vocab; ++x) {
       const float v = to_float(rowp[x]);
       if (v >= bound) a.offer(v, x);
     }
   }
-
-  warp_merge(a);
-  if (lane == 0) {
-    s_part[warp].e = a.seen ? a.e : -CUDART_INF_F;
-    s_part[warp].s = a.s;
+  // The lanes that found something (a handful per block) put their entries into a small pool in
+  // shared memory.  If the pool would overflow (heavy ties: many values equal to the bound), the
+  // lists are merged by shuffles instead, which is slower but has no capacity.
+  {
+    int n_mine = 0;
 #pragma unroll
-    for (int j = 0; j < K; ++j) { s_part[warp].v[j] = a.v[j]; s_part[warp].i[j] = a.i[j]; }
+    for (int j = 0; j < K; ++j) n_mine += a.i[j] != INT_MAX;
+    if (n_mine > 0) {
+      const int at = atomicAdd(&s_cnt, n_mine);
+      if (at + n_mine <= kPoolCap) {
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+          if (j < n_mine) { s_pool_v[at + j] = a.v[j]; s_pool_i[at + j] = a.i[j]; }
+      }
+    }
   }
   __syncthreads();
-  if (warp != 0) return;
-  a.init();
-  if (lane < kTopkWarps) {
-    a.seen = s_part[lane].e != -CUDART_INF_F;
-    a.e = a.seen ? s_part[lane].e : 0.f;
-    a.s = s_part[lane].s;
+  const int n_pool = s_cnt;
+  if (n_pool > kPoolCap) {
+    a.seen = m != -CUDART_INF_F;
+    a.e = e;
+    a.s = s;
+    warp_merge(a);
+    if (lane == 0) {
+      s_part[warp].e = a.seen ? a.e : -CUDART_INF_F;
+      s_part[warp].s = a.s;
 #pragma unroll
-    for (int j = 0; j < K; ++j) { a.v[j] = s_part[lane].v[j]; a.i[j] = s_part[lane].i[j]; }
+      for (int j = 0; j < K; ++j) { s_part[warp].v[j] = a.v[j]; s_part[warp].i[j] = a.i[j]; }
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    a.init();
+    if (lane < kTopkWarps) {
+      a.seen = s_part[lane].e != -CUDART_INF_F;
+      a.e = a.seen ? s_part[lane].e : 0.f;
+      a.s = s_part[lane].s;
+#pragma unroll
+      for (int j = 0; j < K; ++j) { a.v[j] = s_part[lane].v[j]; a.i[j] = s_part[lane].i[j]; }
+    }
+    warp_merge(a);
+  } else {
+    if (warp != 0) return;
+    // sum of the warps' sums (fixed tree), and the pool's best K by rank: every lane counts the
+    // entries that come before its own (keys are unique), so rank r goes to slot r without a sort
+    float st = lane < kTopkWarps ? s_wsum[lane] : 0.f;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) st += __shfl_xor_sync(0xffffffffu, st, off);
+    if (lane < K) { s_res_v[lane] = -CUDART_INF_F; s_res_i[lane] = INT_MAX; }
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < kPoolCap / 32; ++h) {
+      const int q = lane + 32 * h;
+      if (q < n_pool) {
+        const float v = s_pool_v[q];
+        const int i = s_pool_i[q];
+        int rank = 0;
+        for (int o = 0; o < n_pool; ++o) rank += key_before(s_pool_v[o], s_pool_i[o], v, i);
+        if (rank < K) { s_res_v[rank] = v; s_res_i[rank] = i; }
+      }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < K; ++j) { a.v[j] = s_res_v[j]; a.i[j] = s_res_i[j]; }
+    a.seen = M != -CUDART_INF_F;
+    a.e = E;
+    a.s = st;
   }
-  warp_merge(a);
   if (n_seg == 1) {
-    if (lane == 0) finalize(a, k, row, conf, topk_idx, topk_prob, lse);
+    finalize(a, k, row, lane, conf, topk_idx, topk_prob, lse);
     return;
   }
   // several segments per row: publish this one, the last to arrive merges all of them
-  unsigned ticket = 0;
+  bool last = false;
   if (lane == 0) {
     Partial<K>* p = partials + row * n_seg + seg;
     p->e = a.seen ? a.e : -CUDART_INF_F;
@@ -435,11 +500,10 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
 #pragma unroll
     for (int j = 0; j < K; ++j) { p->v[j] = a.v[j]; p->i[j] = a.i[j]; }
     __threadfence();
-    ticket = atomicInc(tickets + row, (unsigned)(n_seg - 1));  // wraps back to 0 after n_seg arrivals
+    last = ticket_arrive(tickets + row, n_seg);
     __threadfence();
   }
-  ticket = __shfl_sync(0xffffffffu, ticket, 0);
-  if (ticket != (unsigned)(n_seg - 1)) return;
+  if (!__shfl_sync(0xffffffffu, last, 0)) return;
   a.init();
   if (lane < n_seg) {
     const Partial<K>* p = partials + row * n_seg + lane;
@@ -451,7 +515,7 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     for (int j = 0; j < K; ++j) { a.v[j] = __ldcg(&p->v[j]); a.i[j] = __ldcg(&p->i[j]); }
   }
   warp_merge(a);
-  if (lane == 0) finalize(a, k, row, conf, topk_idx, topk_prob, lse);
+  finalize(a, k, row, lane, conf, topk_idx, topk_prob, lse);
 }
 
 struct TopkPlan {
@@ -494,10 +558,6 @@ static cudaError_t launch_topk(const void* logits, int64_t n_rows, int vocab, in
                                void* ws, cudaStream_t st) {
   Partial<K>* partials = reinterpret_cast<Partial<K>*>(ws);
   unsigned* tickets = reinterpret_cast<unsigned*>(static_cast<char*>(ws) + p.ticket_off);
-  if (p.n_seg > 1) {
-    cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)n_rows * 4, st);
-    if (e != cudaSuccess) return e;
-  }
   if (p.threads == 512)
     confidence_topk_kernel<T, K, 512><<<(unsigned)(n_rows * p.n_seg), 512, 0, st>>>(
         static_cast<const T*>(logits), vocab, row_stride, k, p.n_seg, p.chunks_per_seg, conf, idx, prob,
@@ -634,8 +694,9 @@ extern "C" int tsd_confidence_topk_static(const void* logits, int32_t dtype, int
     cudaError_t e = tsd::static_scratch_address(&scratch);
     if (e != cudaSuccess) return tsd::cuda_fail(e, "cudaGetSymbolAddress(g_topk_scratch)");
   }
-  // the launcher zeroes the ticket words inside the scratch on the stream before the kernel; the
-  // partial-result slots are fully rewritten by every call that reads them
+  // ticket words need no clearing (a word that does not carry the in-use tag counts as idle, and
+  // the last arrival of a row returns it to idle); the partial-result slots are fully rewritten by
+  // every call that reads them
   cudaError_t e = dtype == TSD_F32
       ? tsd::dispatch_k<float>(p.K, logits, n_rows, vocab, row_stride, k, p, conf, topk_idx, topk_prob,
                                lse, scratch, stream)

@@ -310,6 +310,43 @@ def test_topk_minus_inf_and_split_rows():
     assert idx[0].tolist() == [77, 0, 1, 2] and prob[0, 1] == 0
 
 
+@pytest.mark.parametrize("fill", ["ones", "random", "last_call"])
+def test_topk_workspace_needs_no_clearing(fill):
+    # few rows: each row is split over several blocks that meet through ticket words in the
+    # workspace; whatever the workspace held before (all bits set, noise, the previous call's
+    # leftovers), the results are the oracle's
+    V, k = 50000, 3
+    g = torch.Generator(device=DEV).manual_seed(11)
+    x = (torch.randn((5, V), generator=g, device=DEV) * 3).bfloat16()
+    nbytes = B.tsd_confidence_topk_workspace_bytes(5, V, k)
+    assert nbytes > 0
+    if fill == "ones":
+        ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device=DEV)
+    else:
+        ws = torch.randint(0, 256, (nbytes,), generator=g, device=DEV, dtype=torch.uint8)
+    r_conf, r_idx, r_prob, _ = oracle.confidence_topk(_np(x), k)
+    for call in range(3 if fill == "last_call" else 1):
+        conf = torch.zeros(5, dtype=torch.float32, device=DEV)
+        idx = torch.zeros((5, k), dtype=torch.int32, device=DEV)
+        prob = torch.zeros((5, k), dtype=torch.float32, device=DEV)
+        B.tsd_confidence_topk(x, k, conf, idx, prob, None, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(idx.cpu().numpy(), r_idx)
+        assert np.abs(conf.cpu().numpy() - r_conf).max() <= 1e-5
+        assert np.abs(prob.cpu().numpy() - r_prob).max() <= 1e-5
+
+
+def test_topk_all_equal_rows_whole_and_split():
+    # every value ties with the bound: far more candidates than the block's candidate pool holds,
+    # so the lowest indices must come out of the slower merge path, for whole and for split rows
+    for n, V in ((3, 126464), (200, 30000), (2, 777)):
+        x = torch.full((n, (V + 7) // 8 * 8), 1.5, dtype=torch.bfloat16, device=DEV)[:, :V]
+        x[0, V // 2:] = 2.0          # the upper half of row 0 ties at a higher value
+        conf, idx, prob = _check_topk(x, 4)
+        assert idx[0].tolist() == [V // 2 + j for j in range(4)]
+        assert idx[1].tolist() == [0, 1, 2, 3]
+
+
 def test_topk_is_deterministic():
     cfg = W.CONFIGS["cfg2"]
     vi = W.verify_inputs(cfg, DEV)
