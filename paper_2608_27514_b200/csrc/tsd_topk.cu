@@ -8,7 +8,7 @@
 //      one multiply, adds 2^(x*log2e - e) for every value (one FFMA + one ex2 each), and stores the
 //      batch maximum in shared memory.
 //   2. bound: the k-th largest of the warps' maxima (one shuffle reduction per warp, then every
-//      thread selects among the 8 or 16 values in registers).  At least k values of the row are
+//      warp ranks the 8 or 16 values, one per lane).  At least k values of the row are
 //      >= it, so it is a valid lower bound of the k-th best.
 //   3. collect: each warp re-reads only those of its batches whose maximum reaches the bound
 //      (a handful per row, served by L2); the values >= bound go into a small pool in shared
@@ -349,9 +349,8 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
   }
 
   // ---- phase 2: bound = k-th largest of the warps' maxima.  Each of the k best warps holds a
-  // value equal to its maximum, so at least k values of the piece reach the bound.  One shuffle
-  // reduction per warp; after the block-wide barrier every thread picks the k-th largest of the
-  // WARPS values in registers (no further shuffles or barriers).
+  // value equal to its maximum, so at least k values of the segment reach the bound.  One shuffle
+  // reduction per warp, one block-wide barrier, then a rank count per warp.
   if (tid == 0) s_cnt = 0;
   {
     float wm = m;
@@ -360,29 +359,22 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     if (lane == 0) s_wmax[warp] = wm;
   }
   __syncthreads();
-  float M = -CUDART_INF_F, bound = -CUDART_INF_F;
+  // lane l < WARPS takes warp maximum l and counts the maxima that come before it (larger, or
+  // equal from a lower warp): ranks are unique, rank 0 is the block maximum, rank K-1 the bound
+  float M, bound;
   {
-    float wv[kTopkWarps];
+    const float mine = lane < kTopkWarps ? s_wmax[lane] : -CUDART_INF_F;
+    int rank = 0;
 #pragma unroll
-    for (int q = 0; q < kTopkWarps / 4; ++q) {
-      const float4 f = reinterpret_cast<const float4*>(s_wmax)[q];
-      wv[4 * q] = f.x; wv[4 * q + 1] = f.y; wv[4 * q + 2] = f.z; wv[4 * q + 3] = f.w;
+    for (int q = 0; q < kTopkWarps; ++q) {
+      const float o = s_wmax[q];
+      rank += (o > mine || (o == mine && q < lane)) ? 1 : 0;
     }
-#pragma unroll
-    for (int r = 0; r < K; ++r) {
-      float x = wv[0];
-#pragma unroll
-      for (int q = 1; q < kTopkWarps; ++q) x = fmaxf(x, wv[q]);
-      if (r == 0) M = x;
-      bound = x;
-      bool gone = false;  // one instance leaves per round: the k-th largest counts multiplicity
-#pragma unroll
-      for (int q = 0; q < kTopkWarps; ++q) {
-        const bool hit = !gone && wv[q] == x;
-        wv[q] = hit ? -CUDART_INF_F : wv[q];
-        gone = gone || hit;
-      }
-    }
+    const bool in = lane < kTopkWarps;
+    const unsigned b0 = __ballot_sync(0xffffffffu, in && rank == 0);
+    const unsigned bk = __ballot_sync(0xffffffffu, in && rank == K - 1);
+    M = __shfl_sync(0xffffffffu, mine, __ffs(b0) - 1);
+    bound = __shfl_sync(0xffffffffu, mine, __ffs(bk) - 1);
   }
   // the block's sum on the block's exponent base; the per-warp sums meet after the next barrier
   const float E = (M == -CUDART_INF_F) ? 0.f : M * kLog2e;
