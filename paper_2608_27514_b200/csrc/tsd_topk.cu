@@ -312,8 +312,15 @@ confidence_topk_kernel(const T* __restrict__ logits, int vocab, int64_t row_stri
     m = m_new;
     e = e_new;
     float part[kTopkUnroll];  // independent partial sums keep the dependent add chains short
+    if ((it + 1) * kTopkBatch <= c1 - c0) {
 #pragma unroll
-    for (int u = 0; u < kTopkUnroll; ++u) part[u] = Unpack<T>::sum_exp(buf[u], -e, 0.f);
+      for (int u = 0; u < kTopkUnroll; ++u) part[u] = Unpack<T>::sum_exp(buf[u], -e, 0.f);
+    } else {  // the segment's last, partly filled batch: no exponentials for the padding
+      const int base = c0 + it * kTopkBatch + tid;
+#pragma unroll
+      for (int u = 0; u < kTopkUnroll; ++u)
+        part[u] = base + u * kTopkThreads < c1 ? Unpack<T>::sum_exp(buf[u], -e, 0.f) : 0.f;
+    }
     s += (part[0] + part[1]) + (part[2] + part[3]);
   };
   // Optional L2 prefetch `prefetch` batches ahead of the register loads, one 128-byte line per
