@@ -30,10 +30,10 @@ ROTATE_BYTES = 640 * 1024 * 1024  # rotate through input copies at least this la
 # profiles/ (kernel -> workload -> bytes); None where no capture exists.
 NCU_TRAFFIC = {
     # cfg2: measured on this workload (the launch-list capture under profiles/).  Others: the 2048-row
-    # capture (523.9 MB, the top-k capture under profiles/) scaled by logit bytes,
+    # capture (524.7 MB, the top-k capture under profiles/) scaled by logit bytes,
     # traffic being proportional to them.
-    "confidence_topk": {"cfg2": 64.8e6, "cfg3": 523.9e6 * 1024 / 2048, "cfg4": 523.9e6 * 16384 / 2048,
-                        "cfg5": 523.9e6 * 16384 / 2048 * 152064 / 126464},
+    "confidence_topk": {"cfg2": 64.8e6, "cfg3": 524.7e6 * 1024 / 2048, "cfg4": 524.7e6 * 16384 / 2048,
+                        "cfg5": 524.7e6 * 16384 / 2048 * 152064 / 126464},
     # cfg2: measured on this workload; cfg4: the 4-sequence capture (223.4 MB) x 4; cfg5: an earlier
     # 1-sequence capture (49.6 MB, part of the output still in L2) x 4
     # (the attention capture under profiles/).
