@@ -63,6 +63,32 @@ bool attention_tc_supported(const AttnArgs& a);
 size_t attention_tc_workspace_bytes(const tsd_layout& L);
 int launch_attention_tc(const AttnArgs& a);
 
+// ---- ticket words: blocks that share a result meet without waiting for each other ----
+// Each block publishes its part, then arrives on the ticket word; the last arrival reads the
+// others' parts and finishes the result.  A word in use carries kTicketTag in its upper 24 bits
+// and the number of arrivals so far in the lower 8; any other content counts as idle and the last
+// arrival writes 0, so the memory that holds the words needs no clearing between calls.
+constexpr unsigned kTicketTag = 0x7FC3A9u;
+
+#ifdef __CUDACC__
+// One arrival; true for the last of n arrivals (n <= 255).
+__device__ __forceinline__ bool ticket_arrive(unsigned* t, int n) {
+  unsigned old = *reinterpret_cast<volatile unsigned*>(t), assumed, cnt;
+  do {
+    assumed = old;
+    cnt = (assumed >> 8) == kTicketTag ? (assumed & 0xffu) : 0u;
+    const unsigned next = (cnt + 1 == (unsigned)n) ? 0u : ((kTicketTag << 8) | (cnt + 1));
+    old = atomicCAS(t, assumed, next);
+  } while (old != assumed);
+  return cnt + 1 == (unsigned)n;
+}
+// Arrivals so far (a snapshot: more may follow at any time).
+__device__ __forceinline__ unsigned ticket_count(const unsigned* t) {
+  const unsigned v = *reinterpret_cast<const volatile unsigned*>(t);
+  return (v >> 8) == kTicketTag ? (v & 0xffu) : 0u;
+}
+#endif
+
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ __forceinline__ void from_float(float& d, float x) { d = x; }

@@ -32,7 +32,6 @@ constexpr int kTopkUnroll = 4;            // chunks per thread per batch
 constexpr int kTopkSegChunks = 32768;     // chunks per segment at most (batch maxima: 32 KB of smem)
 constexpr int kMaxSegments = 32;
 constexpr int kPoolCap = 64;              // candidate pool of a block (entries)
-constexpr unsigned kTicketTag = 0x7FC3A9u;  // upper 24 bits of a ticket word that is in use
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ bool key_before(float va, int ia, float vb, int ib) {
@@ -183,20 +182,6 @@ __device__ __forceinline__ void finalize(const Acc<K>& a, int k, int64_t row, in
     }
   }
   if (lse && lane == 0) lse[row] = M + logf(Z);
-}
-
-// One arrival on a row's ticket word; true for the last of n_seg arrivals, which also returns the
-// word to idle.  A word in use carries kTicketTag in its upper 24 bits and the number of arrivals
-// so far in the lower 8; any other content counts as idle, so the workspace needs no clearing.
-__device__ __forceinline__ bool ticket_arrive(unsigned* t, int n_seg) {
-  unsigned old = *reinterpret_cast<volatile unsigned*>(t), assumed, cnt;
-  do {
-    assumed = old;
-    cnt = (assumed >> 8) == kTicketTag ? (assumed & 0xffu) : 0u;
-    const unsigned next = (cnt + 1 == (unsigned)n_seg) ? 0u : ((kTicketTag << 8) | (cnt + 1));
-    old = atomicCAS(t, assumed, next);
-  } while (old != assumed);
-  return cnt + 1 == (unsigned)n_seg;
 }
 
 template <typename T>
