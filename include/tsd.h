@@ -201,8 +201,11 @@ int tsd_verify_attention_fp8_cache(const tsd_layout* layout, const void* mask, c
  *   conf       device fp32 [n_rows];  topk_idx device int32 [n_rows, k];
  *   topk_prob  device fp32 [n_rows, k];  lse device fp32 [n_rows], nullable.
  *   workspace  device, 16-byte aligned, tsd_confidence_topk_workspace_bytes()
- *              bytes: per-segment partial results when a row is split across
- *              thread blocks (few rows); 0 bytes when it is not.
+ *              bytes: per-segment partial results and per-row ticket words when
+ *              a row is split across thread blocks (few rows); 0 bytes when it
+ *              is not.  Scratch: it needs no initialisation and can be reused
+ *              by later calls; two calls that may overlap on the GPU need a
+ *              workspace each.
  * ------------------------------------------------------------------------- */
 size_t tsd_confidence_topk_workspace_bytes(int64_t n_rows, int32_t vocab, int32_t k);
 int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32_t vocab,
