@@ -26,6 +26,7 @@ constexpr int kMaxRows = 128;
 constexpr int kRowWords = kMaxRows / 32;
 constexpr int kAcceptThreads = 256;      // a warp per node up to 8 nodes ...
 constexpr int kAcceptMaxThreads = 1024;  // ... and up to 32 warps for larger trees (nodes are taken in turn)
+constexpr int kStageCells = 4096;        // trees of up to this many (node, row) cells are staged in shared memory
 
 struct RelaxedArgs {
   int topk_m;           // candidates per row that count for TSD_ACCEPT_TOPK
@@ -52,6 +53,11 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   __shared__ int s_pl[kMaxBranches];  // prefix_len, kept on chip for the walk (global reads of values
                                       // just written would cost one L2 round trip per node)
   __shared__ int s_acc;
+  // Small trees: every warp loads its node's tokens and top-1 candidates once, together with the
+  // confidences, and the later phases (the parent's rows for the edge test, the accepted node's
+  // candidates for the unmask set) read them from here instead of making two more dependent round
+  // trips to global memory.
+  __shared__ int32_t s_st[kStageCells], s_t1[kStageCells];
   const int s = blockIdx.x, tree = blockIdx.y, batch = gridDim.x;
   const int lo = tree ? n_cur : 0;          // first branch of this tree = its root
   const int B = tree ? B_all - n_cur : n_cur;  // its size (0: nothing to verify)
@@ -63,9 +69,12 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   const float* cf = conf + ((size_t)s * B_all + lo) * R;
   const int32_t* t1 = top1 + ((size_t)s * B_all + lo) * R * top1_stride;
   const int words = min((R + 31) / 32, WORDS);
+  const bool staged = B * R <= kStageCells;
 
   // decode rule U(p) for every node
   for (int p = warp; p < B; p += n_warps) {
+    // the node's parent is requested together with its rows (one address for the whole warp)
+    const int raw_parent = p > 0 ? parent[(size_t)s * B_all + lo + p] : -1;  // forest index
     uint32_t hi[WORDS], any_hi = 0, any_masked = 0;
     float best = -CUDART_INF_F;
     int best_r = INT_MAX;
@@ -76,7 +85,12 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
         const int r = w * 32 + lane;
         bool masked = false, high = false;
         if (r < R) {
-          masked = st[p * R + r] == mask_id;
+          const int32_t tok = st[p * R + r];
+          if (staged) {
+            s_st[p * R + r] = tok;
+            s_t1[p * R + r] = t1[(size_t)(p * R + r) * top1_stride];
+          }
+          masked = tok == mask_id;
           const float c = cf[p * R + r];
 
           high = masked && c > tau;  // strictly above the threshold
@@ -103,10 +117,7 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
 #pragma unroll
       for (int w = 0; w < WORDS; ++w) s_u[p][w] = hi[w];
       int par = -1;
-      if (p > 0) {
-        const int raw = parent[(size_t)s * B_all + lo + p];  // forest index
-        par = raw >= lo ? raw - lo : -1;                      // local to the tree
-      }
+      if (p > 0) par = raw_parent >= lo ? raw_parent - lo : -1;  // local to the tree
       if (p > 0 && (par < 0 || par >= p)) {
         if (status) atomicOr(status, TSD_STATUS_BAD_PARENT);
         par = -1;  // treated as an invalid edge hanging off nothing
@@ -125,7 +136,8 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
       if (r < R) {
         float pr = 0.f;  // probability of the token this child adds at r, under its parent
         if (c > 0 && p >= 0) {
-          const int sp = st[p * R + r], sc = st[c * R + r];
+          const int sp = staged ? s_st[p * R + r] : st[p * R + r];
+          const int sc = staged ? s_st[c * R + r] : st[c * R + r];
           const bool p_masked = sp == mask_id, c_masked = sc == mask_id;
           const bool in_u = (s_u[p][w] >> lane) & 1u;
           if (!p_masked) {
@@ -135,7 +147,7 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
           } else {
             delta = true;
             const int32_t* cand = t1 + (size_t)(p * R + r) * top1_stride;
-            bool tok_ok = cand[0] == sc;
+            bool tok_ok = (staged ? s_t1[p * R + r] : cand[0]) == sc;
             if (rule == TSD_ACCEPT_TOPK)
               for (int j = 1; j < x.topk_m; ++j) tok_ok |= cand[j] == sc;
             if (x.logits && sc >= 0 && sc < x.vocab) {
@@ -203,12 +215,16 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
     for (int w = 0; w < words; ++w) {
       const int r = w * 32 + lane;
       bool f0 = false, fa = false;
-      if (r < R) { f0 = st[r] != mask_id; fa = st[acc * R + r] != mask_id; }
+      if (r < R) {
+        f0 = (staged ? s_st[r] : st[r]) != mask_id;
+        fa = (staged ? s_st[acc * R + r] : st[acc * R + r]) != mask_id;
+      }
       gained += __popc(__ballot_sync(full, fa)) - __popc(__ballot_sync(full, f0));
       if (r < R) {
         const bool in_u = (s_u[acc][w] >> lane) & 1u;
         unmask_flag[ts * R + r] = in_u ? 1 : 0;
-        unmask_tok[ts * R + r] = in_u ? t1[(size_t)(acc * R + r) * top1_stride] : -1;
+        unmask_tok[ts * R + r] =
+            in_u ? (staged ? s_t1[acc * R + r] : t1[(size_t)(acc * R + r) * top1_stride]) : -1;
       }
     }
     if (lane == 0) n_new_tokens[ts] = gained;
