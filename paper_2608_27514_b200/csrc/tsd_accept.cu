@@ -3,7 +3,7 @@
 //
 // One thread block per sequence.  Warps take tree nodes in turn: first the decode rule U(p) of
 // every node (what threshold decoding would unmask next), then the validity of every edge, both
-// as warp ballots over the block's rows; one thread then walks the tree (a few dozen nodes).
+// as warp ballots over the block's rows; one warp then walks the tree, a lane per node.
 // Integer and float compares only: the result is exact.
 //
 // Besides the exact and top-1 tests, the two relaxed readings of the verification test
@@ -171,40 +171,54 @@ accept_kernel(int B_all, int n_cur, int R, const int32_t* __restrict__ parent, c
   }
   __syncthreads();
 
-  // tree walk (parents precede children, so one ascending sweep fills depth and prefix length)
-  if (threadIdx.x == 0) {
-    // a node's depth is found by walking its parents (trees are a few levels deep)
+  // tree walk by warp 0, a lane per node: the lane climbs from its node to the root (trees are a few
+  // levels deep), counting the steps (= depth) and remembering the invalid edge nearest the root;
+  // the leading valid edges on the path root -> node are the ones above that edge.
+  if (warp == 0) {
     int32_t* pl = prefix_len + (size_t)s * B_all + lo;
     uint8_t* ev = edge_valid + (size_t)s * B_all + lo;
-    int acc = 0, acc_depth = 0;
-    s_pl[0] = 0;
-    pl[0] = 0;
-    ev[0] = 1;
-    for (int b = 1; b < B; ++b) {
-      const int p = s_par[b];
-      ev[b] = s_valid[b];
-      int depth_p = 0;
-      for (int a = p; a > 0; a = s_par[a]) ++depth_p;
-      const int plp = p >= 0 ? s_pl[p] : 0;
-      const bool whole = p >= 0 && plp == depth_p && s_valid[b];
-      const int plb = whole ? depth_p + 1 : plp;
+    int best_depth = 0, best_node = 0;  // longest fully valid path seen by this lane (root: depth 0)
+    for (int b = lane; b < B; b += 32) {
+      int depth = 0, bad_at = -1;  // bad_at: steps from b up to the child end of that invalid edge
+      for (int a = b; a > 0; a = s_par[a]) {
+        if (!s_valid[a]) bad_at = depth;
+        ++depth;
+      }
+      const int plb = bad_at < 0 ? depth : depth - bad_at - 1;
       s_pl[b] = plb;
       pl[b] = plb;
-      if (search == TSD_SEARCH_LONGEST && whole && depth_p + 1 > acc_depth) { acc = b; acc_depth = depth_p + 1; }
+      ev[b] = b == 0 ? 1 : s_valid[b];
+      if (bad_at < 0 && depth > best_depth) { best_depth = depth; best_node = b; }  // nodes ascend per lane
     }
-    if (search == TSD_SEARCH_GREEDY) {
+    int acc = 0, acc_depth = 0;
+    if (search == TSD_SEARCH_LONGEST) {
+      // deepest fully valid node, lowest index among equals
+#pragma unroll
+      for (int off = 16; off; off >>= 1) {
+        const int od = __shfl_xor_sync(full, best_depth, off), on = __shfl_xor_sync(full, best_node, off);
+        if (od > best_depth || (od == best_depth && on < best_node)) { best_depth = od; best_node = on; }
+      }
+      acc = best_node;
+      acc_depth = best_depth;
+    } else {
+      // greedy: from the root, keep moving to the lowest-index valid child
       for (;;) {
         int next = -1;
-        for (int b = acc + 1; b < B; ++b)
-          if (s_par[b] == acc && s_valid[b]) { next = b; break; }
+        for (int b0 = 0; b0 < B && next < 0; b0 += 32) {
+          const int b = b0 + lane;
+          const unsigned m = __ballot_sync(full, b < B && b > acc && s_par[b] == acc && s_valid[b]);
+          if (m) next = b0 + __ffs(m) - 1;
+        }
         if (next < 0) break;
         acc = next;
         ++acc_depth;
       }
     }
-    accepted_node[ts] = lo + acc;  // index in the forest
-    accepted_len[ts] = acc_depth;
-    s_acc = acc;
+    if (lane == 0) {
+      accepted_node[ts] = lo + acc;  // index in the forest
+      accepted_len[ts] = acc_depth;
+      s_acc = acc;
+    }
   }
   __syncthreads();
 
