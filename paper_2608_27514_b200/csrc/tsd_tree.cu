@@ -41,16 +41,22 @@ __device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {  // 
   if (a.row != b.row) return a.row < b.row;
   return a.rank < b.rank;
 }
+// The best candidate of the warp in two warp-wide reductions (redux.sync): probabilities are
+// non-negative, so their bit patterns order like unsigned integers; among the lanes that hold the
+// largest one, the smallest (row, rank) wins.  Every lane returns with the winner.
 __device__ __forceinline__ Cand warp_best(Cand c) {
-#pragma unroll
-  for (int off = 16; off; off >>= 1) {
-    Cand o;
-    o.p = __shfl_xor_sync(0xffffffffu, c.p, off);
-    o.row = __shfl_xor_sync(0xffffffffu, c.row, off);
-    o.rank = __shfl_xor_sync(0xffffffffu, c.rank, off);
-    if (cand_before(o, c)) c = o;
-  }
-  return c;
+  const unsigned full = 0xffffffffu;
+  const bool valid = c.row >= 0 && c.p >= 0.f;
+  const unsigned pk = valid ? (c.p > 0.f ? __float_as_uint(c.p) + 1u : 1u) : 0u;  // 0 = no candidate in this lane
+  const unsigned pmax = __reduce_max_sync(full, pk);
+  Cand w = {0.f, -1, 0};
+  if (pmax == 0u) return w;
+  const unsigned rr = (valid && pk == pmax) ? ((unsigned)c.row << 8) | (unsigned)c.rank : 0xffffffffu;
+  const unsigned rmin = __reduce_min_sync(full, rr);
+  w.p = __uint_as_float(pmax - 1u);  // a zero of either sign comes back as +0
+  w.row = (int)(rmin >> 8);
+  w.rank = (int)(rmin & 0xffu);
+  return w;
 }
 
 // RPL = rows per lane (R <= 32 * RPL), KK = candidates per row held in registers (k <= KK): the
