@@ -430,6 +430,55 @@ def test_accept_random_trees_match_oracle(R):
             assert B.tsd_check_status(status) == B.TSD_OK
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_accept_random_shapes_chains_and_broken_parents(seed):
+    # tree sizes and block lengths drawn at random, up to the limits (256 nodes, 128 rows); some
+    # trees are long chains (the walk climbs many levels), some have parents that point nowhere
+    # (an invalid edge hanging off nothing, whose descendants inherit a prefix of 0)
+    rng = np.random.default_rng(9000 + seed)
+    R = int(rng.choice([1, 4, 31, 32, 33, 64, 100, 128]))
+    Bn = int(rng.choice([1, 2, 5, 8, 33, 64, 130, 256]))
+    S, V = int(rng.integers(1, 6)), 50
+    M = V
+    deep = seed % 3 == 0
+    parent = np.stack([[-1] + [int(b - 1 if deep and rng.random() < 0.8 else rng.integers(0, b))
+                               for b in range(1, Bn)] for _ in range(S)]).astype(np.int32)
+    broken = seed % 2 == 1 and Bn > 2
+    if broken:
+        for s in range(S):
+            for b in rng.integers(1, Bn, 2):
+                parent[s, b] = int(rng.choice([-1, b, b + 3, -5]))
+    conf = rng.random((S, Bn, R)).astype(np.float32)
+    conf[rng.random((S, Bn, R)) < 0.2] = 0.8
+    top1 = rng.integers(0, V, (S, Bn, R)).astype(np.int32)
+    state = np.full((S, Bn, R), M, np.int32)
+    for s in range(S):
+        fill = rng.random(R) < 0.3
+        state[s, 0, fill] = rng.integers(0, V, fill.sum())
+        for b in range(1, Bn):
+            p = parent[s, b] if 0 <= parent[s, b] < b else 0
+            c = state[s, p].copy()
+            flag, tok = oracle.decode_rule(state[s, p], M, conf[s, p], top1[s, p], 0.8)
+            mode = rng.integers(0, 5)
+            rows = np.flatnonzero(c == M)
+            if mode <= 2:
+                c[flag.astype(bool)] = tok[flag.astype(bool)]
+            elif mode == 3 and len(rows):
+                r = rows[rng.integers(len(rows))]
+                c[r] = top1[s, p, r]
+            elif len(rows):
+                c[rows[0]] = rng.integers(0, V)
+            state[s, b] = c
+    for rule in (0, 1):
+        for search in (0, 1):
+            ref = oracle.accept(parent, state, M, conf, top1, 0.8, rule, search)
+            got, status = _gpu_accept(parent, state, M, conf, top1, 0.8, rule, search)
+            for key, val in ref.items():
+                assert np.array_equal(got[key], val), (key, rule, search)
+            want = B.TSD_ERR_DEVICE_DATA if broken else B.TSD_OK
+            assert B.tsd_check_status(status) == want
+
+
 def test_accept_reports_bad_parent_without_faulting():
     parent = np.array([[-1, 0, 7, 1]], np.int32)       # node 2 points past itself
     state = np.full((1, 4, 32), 9, np.int32)
