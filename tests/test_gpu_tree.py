@@ -41,7 +41,8 @@ def _oracle_tree(prev_state, acc, flag, tok, mask_id, idx, prob, width, depth, m
 
 @pytest.mark.parametrize("R,k,Wd,D,Bn", [(32, 3, 2, 2, 4), (32, 3, 3, 3, 7), (64, 3, 3, 3, 16), (128, 8, 32, 4, 256),
                                           (5, 1, 1, 1, 2), (32, 4, 4, 0, 8), (32, 2, 8, 6, 40)])
-def test_tree_matches_oracle_random_pools(R, k, Wd, D, Bn):
+@pytest.mark.parametrize("lowest", [1, 0])   # 0: candidates of probability exactly zero take part too
+def test_tree_matches_oracle_random_pools(R, k, Wd, D, Bn, lowest):
     rng = np.random.default_rng(R * 1000 + k * 100 + Wd)
     S, Bp, V = 9, 5, 1000
     M = V
@@ -51,7 +52,7 @@ def test_tree_matches_oracle_random_pools(R, k, Wd, D, Bn):
     flag = (rng.random((S, R)) < 0.15).astype(np.uint8)
     tok = rng.integers(0, V, (S, R)).astype(np.int32)
     idx = rng.integers(0, V, (S, Bp, R, k)).astype(np.int32)
-    prob = (rng.integers(1, 64, (S, Bp, R, k)) / 64.0).astype(np.float32)   # coarse values: many ties
+    prob = (rng.integers(lowest, 64 if lowest else 4, (S, Bp, R, k)) / 64.0).astype(np.float32)   # coarse values: many ties
     prob = -np.sort(-prob, axis=-1)
     got = _gpu_tree(prev, acc, flag, tok, M, idx, prob, Wd, D, Bn)
     ref = _oracle_tree(prev, acc, flag, tok, M, idx, prob, Wd, D, Bn)
