@@ -39,13 +39,8 @@ def _run_attention(cfg, attn, flags, vis=None, cache_lens=None, want_dense=False
     return step, dense
 
 
-def _check_attention(cfg, attn, flags, vis=None, cache_lens=None, heads=None, seqs=None):
-    """Compare with the oracle; `heads`/`seqs` restrict the oracle to a sample."""
-    step, dense = _run_attention(cfg, attn, flags, vis, cache_lens, want_dense=True)
-    mask = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc,
-                             None if vis is None else vis.cpu().numpy(),
-                             None if cache_lens is None else cache_lens.cpu().numpy())
-    assert np.array_equal(dense.cpu().numpy(), mask)
+def _compare_attention(step, cfg, attn, mask, heads=None, seqs=None):
+    """`step.out` / `step.attn_lse` against the oracle; `heads`/`seqs` restrict the oracle to a sample."""
     seqs = list(range(cfg.S)) if seqs is None else seqs
     group = cfg.Hq // cfg.Hkv
     kv_heads = list(range(cfg.Hkv)) if heads is None else heads
@@ -65,6 +60,16 @@ def _check_attention(cfg, attn, flags, vis=None, cache_lens=None, heads=None, se
             assert np.abs(got_lse - ref_lse).max() <= (2e-2 if cfg.dtype == "bf16" else 1e-4)
             worst = max(worst, err.max())
     return worst
+
+
+def _check_attention(cfg, attn, flags, vis=None, cache_lens=None, heads=None, seqs=None):
+    """Run the attention stage and compare with the oracle (dense mask bit for bit as well)."""
+    step, dense = _run_attention(cfg, attn, flags, vis, cache_lens, want_dense=True)
+    mask = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc,
+                             None if vis is None else vis.cpu().numpy(),
+                             None if cache_lens is None else cache_lens.cpu().numpy())
+    assert np.array_equal(dense.cpu().numpy(), mask)
+    return _compare_attention(step, cfg, attn, mask, heads, seqs)
 
 
 # ----------------------------------------------------------------------------- mask
@@ -516,6 +521,43 @@ def test_whole_step_matches_oracle(name):
         assert np.array_equal(res[key].cpu().numpy(), own[key]), key
     # the plan the generator planted is what the decoder found
     assert int(res["edge_valid"].sum()) >= S
+
+
+@pytest.mark.parametrize("name,seqs,heads", [("cfg4", [0, 9], [5, 31]), ("cfg5", [2], [1, 3])])
+def test_whole_step_full_size_matches_oracle(name, seqs, heads):
+    # the two large workloads through VerifyStep.run, as the benchmark launches them: the oracle
+    # scores EVERY row of the vocabulary pass (logits streamed to the host in slabs), the
+    # acceptance runs on the full planted trees, attention is compared on sampled (sequence, kv
+    # head) pairs (its fp64 oracle needs minutes for the whole batch)
+    cfg = W.CONFIGS[name]
+    attn = W.attention_inputs(cfg, DEV)
+    vi = W.verify_inputs(cfg, DEV)
+    step = VerifyStep.for_config(cfg, DEV)
+    res = step.run(attn, vi["logits"], vi["parent"], vi["state"], vi["mask_id"], cfg.tau)
+    torch.cuda.synchronize()
+    step.check_status()
+    S, Bn, R = cfg.S, cfg.B, cfg.R
+    g_idx, g_conf, g_prob = step.topk_idx.cpu().numpy(), step.conf.cpu().numpy(), step.topk_prob.cpu().numpy()
+    conf = np.empty(cfg.rows, np.float64)
+    top1 = np.empty(cfg.rows, np.int32)
+    slab = 1024
+    for r0 in range(0, cfg.rows, slab):
+        r1 = min(cfg.rows, r0 + slab)
+        o_conf, o_idx, o_prob, _ = oracle.confidence_topk(_np(vi["logits"][r0:r1]), cfg.k)
+        assert np.array_equal(g_idx[r0:r1], o_idx), "top-k indices, rows %d..%d" % (r0, r1)
+        assert np.abs(g_conf[r0:r1] - o_conf).max() <= 1e-5
+        assert np.abs(g_prob[r0:r1] - o_prob).max() <= 1e-5
+        conf[r0:r1], top1[r0:r1] = o_conf, o_idx[:, 0]
+    parent, state = _np(vi["parent"]), _np(vi["state"])
+    same = oracle.accept(parent, state, vi["mask_id"], g_conf.reshape(S, Bn, R), top1.reshape(S, Bn, R), cfg.tau)
+    own = oracle.accept(parent, state, vi["mask_id"], conf.astype(np.float32).reshape(S, Bn, R),
+                        top1.reshape(S, Bn, R), cfg.tau)
+    for key in same:
+        assert np.array_equal(res[key].cpu().numpy(), same[key]), key
+        assert np.array_equal(res[key].cpu().numpy(), own[key]), key
+    assert int(res["accepted_len"].sum()) > 0            # planted continuations really are accepted
+    mask = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc)
+    _compare_attention(step, cfg, attn, mask, heads=heads, seqs=seqs)
 
 
 def test_topk_subnormal_and_signed_zero_logits():
