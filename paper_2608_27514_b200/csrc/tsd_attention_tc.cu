@@ -175,23 +175,6 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D (tensor memory) (+)= A (tensor memory) x B (shared memory).  ACC is a compile-time constant so
-// that the accumulate predicate costs nothing at issue time.
-template <bool ACC>
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
-  if (ACC)
-    asm volatile("{\n.reg .pred p;\nsetp.eq.b32 p, 0, 0;\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc) : "memory");
-  else
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, 0, 0;\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc) : "memory");
-}
-
 #define TSD_R16(a, o) "=r"(a[o+0]), "=r"(a[o+1]), "=r"(a[o+2]), "=r"(a[o+3]), "=r"(a[o+4]), "=r"(a[o+5]), "=r"(a[o+6]), "=r"(a[o+7]), \
   "=r"(a[o+8]), "=r"(a[o+9]), "=r"(a[o+10]), "=r"(a[o+11]), "=r"(a[o+12]), "=r"(a[o+13]), "=r"(a[o+14]), "=r"(a[o+15])
 #define TSD_W16(a, o) "r"(a[o+0]), "r"(a[o+1]), "r"(a[o+2]), "r"(a[o+3]), "r"(a[o+4]), "r"(a[o+5]), "r"(a[o+6]), "r"(a[o+7]), \
@@ -339,28 +322,59 @@ struct TcParams {
   float scale_log2e;              // sm_scale * log2(e), > 0
 };
 
-// One Q K^T: 8 MMAs (K = 16 over head_dim) into S buffer B, Q from tensor memory at `q_tmem`, K from
-// the stage whose offset (in 16-byte units) is `k_off`.
-template <int B>
-__device__ __forceinline__ void issue_qk_mmas(uint32_t utmem, uint32_t q_tmem, const uint64_t (&kd)[8], uint32_t k_off,
+// The MMAs of a tile go out as ONE block of instructions: the issuing lane shares its scheduler with
+// three softmax warps, so every instruction between two MMAs (a predicate, a 64-bit add for a
+// descriptor) is a gap in which the tensor pipe may run dry.  Descriptors are passed as their low
+// words (the address field varies, the high word is the same for all of one operand).
+//
+// One Q K^T: 8 MMAs (K = 16 over head_dim) into the S buffer at tensor-memory address `s_tmem`, Q
+// from tensor memory at `q_tmem`, K through the descriptors (lo[kk], hi); then the two commits.
+__device__ __forceinline__ void issue_qk_mmas(uint32_t s_tmem, uint32_t q_tmem, const uint32_t (&lo)[8], uint32_t hi,
                                               uint32_t s_full, uint32_t k_free) {
   constexpr uint32_t idesc_qk = instr_desc(kKeys, 0);
-  tc_mma_ts<false>(utmem + kColS + B * kKeys, q_tmem, kd[0] + k_off, idesc_qk);
-#pragma unroll
-  for (int kk = 1; kk < 8; ++kk) tc_mma_ts<true>(utmem + kColS + B * kKeys, q_tmem + kk * 8, kd[kk] + k_off, idesc_qk);
-  tc_commit(s_full);
-  tc_commit(k_free);
+  asm volatile(
+      "{\n.reg .pred pf, pt;\n.reg .b32 a;\n.reg .b64 dsc;\n"
+      "setp.ne.b32 pf, 0, 0;\nsetp.eq.b32 pt, 0, 0;\n"
+      "mov.b64 dsc, {%2, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], dsc, %11, pf;\n"
+      "add.u32 a, %1, 8;\nmov.b64 dsc, {%3, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 16;\nmov.b64 dsc, {%4, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 24;\nmov.b64 dsc, {%5, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 32;\nmov.b64 dsc, {%6, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 40;\nmov.b64 dsc, {%7, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 48;\nmov.b64 dsc, {%8, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "add.u32 a, %1, 56;\nmov.b64 dsc, {%9, %10};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %11, pt;\n"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%12];\n"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%13];\n}"
+      ::"r"(s_tmem), "r"(q_tmem), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]), "r"(lo[4]), "r"(lo[5]), "r"(lo[6]),
+        "r"(lo[7]), "r"(hi), "r"(idesc_qk), "r"(s_full), "r"(k_free) : "memory");
 }
-// One P V: 4 MMAs (16 keys = 8 packed columns of P each) from P buffer VB mod 2 and V stage VB into O.
-template <int VB, bool ACC>
-__device__ __forceinline__ void issue_pv_mmas(uint32_t utmem, const uint64_t (&vd)[kKeys / 16], uint32_t pv_done) {
+// One P V: 4 MMAs (16 keys = 8 packed columns of P each), P from tensor memory at `p_tmem`, V through
+// the descriptors (lo[kk], hi), into O at `o_tmem`; `acc` = 0 starts a new accumulation; then the commit.
+__device__ __forceinline__ void issue_pv_mmas(uint32_t o_tmem, uint32_t p_tmem, const uint32_t (&lo)[kKeys / 16], uint32_t hi,
+                                              uint32_t acc, uint32_t pv_done) {
   constexpr uint32_t idesc_pv = instr_desc(128, 1);
-  constexpr uint64_t stage = (uint64_t)((VB * kKVBytes) >> 4);
-  constexpr uint32_t p_col = kColP + (VB & 1) * 32;
-  tc_mma_ts<ACC>(utmem + kColO, utmem + p_col, vd[0] + stage, idesc_pv);
-#pragma unroll
-  for (int kk = 1; kk < kKeys / 16; ++kk) tc_mma_ts<true>(utmem + kColO, utmem + p_col + kk * 8, vd[kk] + stage, idesc_pv);
-  tc_commit(pv_done);
+  asm volatile(
+      "{\n.reg .pred pa, pt;\n.reg .b32 a;\n.reg .b64 dsc;\n"
+      "setp.ne.b32 pa, %7, 0;\nsetp.eq.b32 pt, 0, 0;\n"
+      "mov.b64 dsc, {%2, %6};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], dsc, %8, pa;\n"
+      "add.u32 a, %1, 8;\nmov.b64 dsc, {%3, %6};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %8, pt;\n"
+      "add.u32 a, %1, 16;\nmov.b64 dsc, {%4, %6};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %8, pt;\n"
+      "add.u32 a, %1, 24;\nmov.b64 dsc, {%5, %6};\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], dsc, %8, pt;\n"
+      "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n}"
+      ::"r"(o_tmem), "r"(p_tmem), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]), "r"(hi), "r"(acc), "r"(idesc_pv),
+        "r"(pv_done) : "memory");
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -544,9 +558,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       long long acc_a = 0, acc_c = 0;
       int sb = 0, kb = 0;   // S buffer of tile G = G mod 3, K stage = G mod 5
       uint32_t kph = 0;     // (G / 5) & 1
-      uint64_t kd[8];  // descriptors of stage 0; the others differ in the address field only
+      uint32_t kd_lo[8];  // low words of the descriptors of K stage 0; the others differ in the address field only
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) kd[kk] = smem_desc(ubase + kOffK + (kk >> 2) * kSubKV + (kk & 3) * 32, 16, 1024);
+      for (int kk = 0; kk < 8; ++kk)
+        kd_lo[kk] = (uint32_t)smem_desc(ubase + kOffK + (kk >> 2) * kSubKV + (kk & 3) * 32, 16, 1024);
+      const uint32_t kd_hi = (uint32_t)(smem_desc(0, 16, 1024) >> 32);
       bool ready = false;  // the barrier of the tile at hand was seen complete by the early test
       for (int it = 0; it < n_run && ok; ++it) {
         const int T = __shfl_sync(0xffffffffu, item_T[it], 0);
@@ -567,12 +583,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const uint32_t kph1 = kb1 == 0 ? kph ^ 1u : kph;
           const bool seen = mbar_test_wait(bar(QK_GO + kb1), kph1);  // used after the MMAs
           if (elect_one()) {
-            const uint32_t k_off = (uint32_t)kb * (kKVBytes >> 4), k_free = bar(K_FREE + kb);
-            switch (sb) {
-              case 0: issue_qk_mmas<0>(utmem, q_tmem, kd, k_off, bar(S_FULL + 0), k_free); break;
-              case 1: issue_qk_mmas<1>(utmem, q_tmem, kd, k_off, bar(S_FULL + 1), k_free); break;
-              default: issue_qk_mmas<2>(utmem, q_tmem, kd, k_off, bar(S_FULL + 2), k_free); break;
-            }
+            const uint32_t k_off = (uint32_t)kb * (kKVBytes >> 4);
+            uint32_t lo[8];
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) lo[kk] = kd_lo[kk] + k_off;
+            issue_qk_mmas(utmem + kColS + (uint32_t)sb * kKeys, q_tmem, lo, kd_hi, bar(S_FULL + sb), bar(K_FREE + kb));
           }
           __syncwarp();
           ready = seen;
@@ -587,9 +602,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (lane == 0) { TSD_TR_SUM(0, 201, acc_a); TSD_TR_SUM(2, 201, acc_c); TSD_TR_SUM(3, 201, (long long)G); }
     } else {
       long long acc_a = 0, acc_c = 0;
-      uint64_t vd[kKeys / 16];
+      uint32_t vd_lo[kKeys / 16];
 #pragma unroll
-      for (int kk = 0; kk < kKeys / 16; ++kk) vd[kk] = smem_desc(ubase + kOffV + kk * 2048, kSubKV, 1024);
+      for (int kk = 0; kk < kKeys / 16; ++kk) vd_lo[kk] = (uint32_t)smem_desc(ubase + kOffV + kk * 2048, kSubKV, 1024);
+      const uint32_t vd_hi = (uint32_t)(smem_desc(0, kSubKV, 1024) >> 32);
       bool ready = false;
       for (int it = 0; it < n_run && ok; ++it) {
         const int T = __shfl_sync(0xffffffffu, item_T[it], 0);
@@ -609,21 +625,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const long long c2 = TSD_CLK();
           const bool seen = mbar_test_wait(bar(PV_GO + ((G + 1) & 3)), ((G + 1) >> 2) & 1);  // used after the MMAs
           if (elect_one()) {
-            if (j == 0) {
-              switch (b) {
-                case 0: issue_pv_mmas<0, false>(utmem, vd, bar(PV_DONE + 0)); break;
-                case 1: issue_pv_mmas<1, false>(utmem, vd, bar(PV_DONE + 1)); break;
-                case 2: issue_pv_mmas<2, false>(utmem, vd, bar(PV_DONE + 2)); break;
-                default: issue_pv_mmas<3, false>(utmem, vd, bar(PV_DONE + 3)); break;
-              }
-            } else {
-              switch (b) {
-                case 0: issue_pv_mmas<0, true>(utmem, vd, bar(PV_DONE + 0)); break;
-                case 1: issue_pv_mmas<1, true>(utmem, vd, bar(PV_DONE + 1)); break;
-                case 2: issue_pv_mmas<2, true>(utmem, vd, bar(PV_DONE + 2)); break;
-                default: issue_pv_mmas<3, true>(utmem, vd, bar(PV_DONE + 3)); break;
-              }
-            }
+            const uint32_t v_off = (uint32_t)b * (kKVBytes >> 4);
+            uint32_t lo[kKeys / 16];
+#pragma unroll
+            for (int kk = 0; kk < kKeys / 16; ++kk) lo[kk] = vd_lo[kk] + v_off;
+            issue_pv_mmas(utmem + kColO, utmem + kColP + (uint32_t)(b & 1) * 32u, lo, vd_hi, j == 0 ? 0u : 1u, bar(PV_DONE + b));
           }
           __syncwarp();
           ready = seen;
