@@ -377,6 +377,38 @@ __device__ __forceinline__ void issue_pv_mmas(uint32_t o_tmem, uint32_t p_tmem, 
         "r"(pv_done) : "memory");
 }
 
+// Rarely executed pieces of the softmax warps, kept out of line so that the loop over the key
+// tiles stays small in the instruction cache.
+// One row of O (128 fp32 columns of this thread's tensor-memory lane) times alpha.
+__device__ __noinline__ void rescale_o_row(uint32_t t_o, float alpha) {
+#pragma unroll 1
+  for (int q4 = 0; q4 < 4; ++q4) {
+    uint32_t ov[32];
+    TSD_TMEM_LD32(ov, 0, t_o + q4 * 32);
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+    TSD_TMEM_ST32(ov, 0, t_o + q4 * 32);
+  }
+}
+// One row of Q: staging buffer (128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7),
+// one sub-tile per half of head_dim) -> 64 columns of this thread's tensor-memory lane, as the A
+// operand of Q K^T (32-bit column i = elements 2i, 2i+1).
+__device__ __noinline__ void copy_q_row(uint32_t q_smem, int r, uint32_t t_q) {
+#pragma unroll 1
+  for (int sub = 0; sub < 2; ++sub) {
+    uint32_t w[32];
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+      const uint32_t a = q_smem + sub * kSub + (uint32_t)r * 128u + ((uint32_t)(ch ^ (r & 7)) << 4);
+      asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                   : "=r"(w[ch * 4]), "=r"(w[ch * 4 + 1]), "=r"(w[ch * 4 + 2]), "=r"(w[ch * 4 + 3]) : "r"(a) : "memory");
+    }
+    TSD_TMEM_ST32(w, 0, t_q + sub * 32);
+  }
+  tmem_wait_st();
+}
+
 __global__ void __launch_bounds__(kTcThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                     const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kd,
@@ -658,20 +690,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = ok && mbar_wait(bar(QS_FULL), it & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) return;
-      uint32_t w[64];
-#pragma unroll
-      for (int sub = 0; sub < 2; ++sub)
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint32_t a = base + kOffQ + sub * kSub + (uint32_t)r * 128u + ((uint32_t)(ch ^ (r & 7)) << 4);
-          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(w[sub * 32 + ch * 4]), "=r"(w[sub * 32 + ch * 4 + 1]), "=r"(w[sub * 32 + ch * 4 + 2]),
-                         "=r"(w[sub * 32 + ch * 4 + 3]) : "r"(a) : "memory");
-        }
-      const uint32_t t_q = t_lane + kColQ + (uint32_t)(it & 1) * 64u;
-      TSD_TMEM_ST32(w, 0, t_q);
-      TSD_TMEM_ST32(w, 32, t_q + 32);
-      tmem_wait_st();
+      copy_q_row(base + kOffQ, r, t_lane + kColQ + (uint32_t)(it & 1) * 64u);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(QT_READY + (it & 1)));
@@ -713,7 +732,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_before();
         __syncwarp();
         // S is in registers: the buffer can take the Q K^T of the tile three ahead (if there is one)
-        if (lane == 0 && Gj + kNSb < n_tiles) mbar_arrive(bar(QK_GO + (Gj + kNSb) % kNK));
+        if (lane == 0 && Gj + kNSb < n_tiles) mbar_arrive(bar(QK_GO + (int)((unsigned)(Gj + kNSb) % (unsigned)kNK)));
 
         // visibility of this tile's 64 keys for this row
         uint32_t cm[2] = {0xffffffffu, 0xffffffffu};
@@ -816,15 +835,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t ov[32];
-            TSD_TMEM_LD32(ov, 0, t_lane + kColO + q4 * 32);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-            TSD_TMEM_ST32(ov, 0, t_lane + kColO + q4 * 32);
-          }
+          rescale_o_row(t_lane + kColO, alpha);
         }
         // P (bf16 pairs) into P buffer pb, free once the P V of tile t-2 has completed:
         // column i = keys 2i (low half), 2i+1
