@@ -478,7 +478,7 @@ def main():
         topk=dict(seconds=t_topk, bound="hbm", roofline_seconds=alg["topk_bytes"] / (pk["hbm_gbs"] * 1e9),
                   frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9),
         accept=dict(seconds=t_acc),
-        accept_relaxed_prob_longest=dict(seconds=t_acc_prob, note="Section 3.3's 'exceed tau' reading with the "
+        accept_relaxed_prob_longest=dict(seconds=t_acc_prob, note="Section 3.3's probability-above-tau reading with the "
                                          "gather of the drafted tokens' probabilities; not part of the step"),
         tree_build_next_step=dict(seconds=t_tree, note="Alg. 1 tree construction (W3 D3) for the next step; not part of the step"),
     )

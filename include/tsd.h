@@ -23,7 +23,15 @@
  *     trapping.  Copy the word back and pass it to tsd_check_status().
  *   - Results are deterministic: the same inputs give the same bits.
  *   - Non-finite inputs: -inf logits are ordered last with probability 0;
- *     NaN anywhere gives unspecified values but never a fault.
+ *     NaN anywhere gives unspecified values but never a fault.  In the
+ *     attention stage, rows that no query row of a 128-row query tile may read
+ *     can hold anything, Inf and NaN included: cached rows at or past
+ *     cache_lens[s] (whatever the unused capacity holds) and draft rows of
+ *     branches that none of the tile's branches may read.  Draft K/V rows that
+ *     SOME row of a query tile may read have to be finite: a masked key gets
+ *     weight exactly 0, but 0 x NaN is NaN, so a non-finite value in one
+ *     branch's V rows makes the outputs of the other branches of that tile
+ *     (the 128 / R branches that share 128 consecutive draft rows) unspecified.
  */
 #ifndef TSD_H_
 #define TSD_H_
@@ -52,13 +60,14 @@ typedef enum { TSD_F32 = 0, TSD_BF16 = 1 } tsd_dtype;
 /* Which draft blocks count as verified (Section 3.3).  EXACT: the rows and
  * tokens a child adds equal the set that threshold decoding would unmask at
  * its parent; this is the test under which Theorem 1 holds.  TOP1: every token
- * the child adds is its parent's top prediction at that row (the literal
- * "tokens match the model's top predictions"; admits trajectory drift). */
+ * the child adds equals its parent's arg-max at that row (the first clause of
+ * the test in Section 3.3, "Verification procedure", taken literally; admits
+ * trajectory drift). */
 typedef enum {
   TSD_ACCEPT_EXACT = 0,
   TSD_ACCEPT_TOP1 = 1,
-  /* The two relaxed readings of the same sentence ("or fall within top-k / exceed tau"), served
-   * by tsd_accept_relaxed only.  TOPK: every token the child adds is among its parent's first
+  /* The two relaxed alternatives the same passage mentions in passing (membership among the
+   * top-k candidates; probability above the threshold), served by tsd_accept_relaxed only.  TOPK: every token the child adds is among its parent's first
    * topk_m candidates at that row.  PROB: every token the child adds has probability > tau
    * (strictly) under its parent's distribution at that row.  Both admit drift. */
   TSD_ACCEPT_TOPK = 2,
@@ -159,6 +168,20 @@ int tsd_verify_attention(const tsd_layout* layout, const void* mask,
                          uint32_t flags, uint32_t* status, tsd_stream_t stream);
 
 /* ---------------------------------------------------------------------------
+ * Diagnostic for the time-out reporting path (no counterpart in the paper).
+ * Every wait inside the attention kernel is bounded: a block whose wait runs out
+ * ORs TSD_STATUS_TIMEOUT into the status word, stops issuing work and returns,
+ * so the context stays usable and tsd_check_status() gives TSD_ERR_TIMEOUT.
+ * This call launches one warp that runs that same bounded wait on a barrier
+ * nothing will ever complete, with a limit of `poll_limit` polls (1..65536; a
+ * few dozen microseconds at most), so that a caller, or a test, can see the
+ * whole path work (kernel returns by itself, status word, decoding) without
+ * making anything hang or fault.
+ *   status   device uint32, required: receives TSD_STATUS_TIMEOUT.
+ * ------------------------------------------------------------------------- */
+int tsd_selftest_bounded_wait(uint32_t* status, uint32_t poll_limit, tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
  * Verify attention over an 8-bit K/V cache.  No counterpart in the paper, which
  * keeps the dual cache in the model's dtype: the cache is stored as e4m3 codes
  * (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) with one
@@ -203,8 +226,13 @@ int tsd_verify_attention_fp8_cache(const tsd_layout* layout, const void* mask, c
  *   workspace  device, 16-byte aligned, tsd_confidence_topk_workspace_bytes()
  *              bytes: per-segment partial results and per-row ticket words when
  *              a row is split across thread blocks (few rows); 0 bytes when it
- *              is not.  Scratch: it needs no initialisation and can be reused
- *              by later calls; two calls that may overlap on the GPU need a
+ *              is not.  Zero it once before its first use (cudaMemsetAsync);
+ *              after that it can be reused by later calls of any shape without
+ *              clearing: a completed call leaves every ticket word it used at 0
+ *              and the next call rewrites the partial slots it reads.  (A word
+ *              counts as a live ticket only if it carries a 24-bit tag, so most
+ *              leftover content is harmless, but only a zeroed buffer is
+ *              guaranteed.)  Two calls that may overlap on the GPU need a
  *              workspace each.
  * ------------------------------------------------------------------------- */
 size_t tsd_confidence_topk_workspace_bytes(int64_t n_rows, int32_t vocab, int32_t k);
@@ -227,9 +255,10 @@ int tsd_confidence_topk(const void* logits, int32_t dtype, int64_t n_rows, int32
  *     TSD_ERR_WORKSPACE and nothing is launched; compare
  *     tsd_confidence_topk_workspace_bytes() with the capacity beforehand, and
  *     fall back to tsd_confidence_topk with your own workspace.
- *   - The first call on each device looks the array's device address up
- *     (cudaGetSymbolAddress, with that device current).  Make that first call
- *     before any stream capture begins.
+ *   - Every call looks the array's device address up (cudaGetSymbolAddress,
+ *     with the device current: a host-side query).  The first lookup on a
+ *     device sets the library's module up there: make that first call before
+ *     any stream capture begins.
  *   - All calls on a device share the one array, and it keeps whatever the
  *     previous call left: a completed call leaves every ticket word it used
  *     idle again and the next call overwrites the partial slots it reads.
@@ -359,8 +388,11 @@ int tsd_build_interblock_vis(int32_t batch, int32_t n_branches, int32_t n_cur, u
  * step_base + n, and step_base moves on by n + 1 (by n if the accepted node had
  * no masked row left).
  *
- *   parent, state   device [batch, B] / [batch, B, R]: the verified tree;
- *   accepted_node   device int32 [batch], nullable (= node 0);
+ *   tree_root       forest index of the tree's root: 0 for a tree of its own; n_cur for the
+ *                   next block's tree of a joint pass (Section 3.4), whose nodes, parents and
+ *                   accepted_node are forest indices (as tsd_accept_joint_trees writes them);
+ *   parent, state   device [batch, B] / [batch, B, R]: the verified tree (or forest);
+ *   accepted_node   device int32 [batch], nullable (= the root);
  *   unmask_flag, unmask_tok   device [batch, R], both or neither;
  *   tokens          device int32, nullable: sequence s occupies tokens[s * seq_stride ...];
  *   block_start     device int32 [batch], nullable (= 0): first position of the block; a
@@ -374,7 +406,7 @@ int tsd_build_interblock_vis(int32_t batch, int32_t n_branches, int32_t n_cur, u
  * A parent chain that leaves the tree sets TSD_STATUS_BAD_PARENT and commits U(root) only.
  * R 1..128, B 1..256.
  * ------------------------------------------------------------------------- */
-int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_branch, int32_t tree_root,
                         const int32_t* parent, const int32_t* state, const int32_t* accepted_node,
                         const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
                         int32_t* tokens, int64_t seq_stride, const int32_t* block_start,
@@ -382,9 +414,43 @@ int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_bran
                         uint32_t* status, tsd_stream_t stream);
 
 /* ---------------------------------------------------------------------------
+ * Hand-over of the accepted node's K/V (Appendix A: the dual cache holds
+ * prefix/suffix K/V for a whole block and is refreshed at block boundaries;
+ * Section 3.1: a verification pass already holds what the next step needs).
+ * The pass has computed draft K/V rows for every node of the tree; the rows of
+ * the accepted node are the block's K/V under the tokens that were kept.  This
+ * call copies them, per layer, to a destination of the caller's (typically the
+ * block's position in that layer's cache) so that a block that has just been
+ * completed need not be recomputed before it serves as cached context.  Whether
+ * to use it or to recompute at the boundary, as the paper does, is the caller's
+ * choice: the copied rows were computed while the block still held masked
+ * positions elsewhere in the tree's other nodes, not in this one, so they are
+ * exact for the accepted node's own content.
+ * For sequence s and r < R:
+ *     out[s, out_row0[s] + r, :, :] = draft[s, accepted_node[s] * R + r, :, :]
+ *
+ *   accepted_node   device int32 [batch], nullable (= node 0), a tree-local index as
+ *                   tsd_accept_trajectories writes it;
+ *   k_draft, v_draft  device [batch, B*R, n_kv_heads, head_dim], element strides d_*;
+ *                   v_draft / v_out both NULL copies K only;
+ *   k_out, v_out    device [batch, out_rows, n_kv_heads, head_dim], element strides o_*;
+ *   out_row0        device int32 [batch], nullable (= 0): first destination row.
+ * All bases 16-byte aligned, strides multiples of 16 bytes, head_dim contiguous and a
+ * multiple of 16 bytes.  A node outside [0, B) or a destination outside
+ * [0, out_rows) sets TSD_STATUS_BAD_INDEX and leaves that sequence unwritten.
+ * ------------------------------------------------------------------------- */
+int tsd_gather_accepted_kv(int32_t batch, int32_t n_branches, int32_t rows_per_branch, int32_t n_kv_heads,
+                           int32_t head_dim, int32_t dtype, const int32_t* accepted_node,
+                           const void* k_draft, const void* v_draft, int64_t d_stride_b,
+                           int64_t d_stride_row, int64_t d_stride_head, void* k_out, void* v_out,
+                           int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head,
+                           const int32_t* out_row0, int32_t out_rows, uint32_t* status,
+                           tsd_stream_t stream);
+
+/* ---------------------------------------------------------------------------
  * Acceptance under any of the four rules (Section 3.3, "Verification
- * procedure": tokens "match the model's top predictions (or fall within top-k /
- * exceed tau)"), for one tree (n_cur = n_branches) or the two trees of a joint
+ * procedure": the exact and top-1 tests, and the top-k-membership and
+ * probability-above-tau alternatives), for one tree (n_cur = n_branches) or the two trees of a joint
  * pass; outputs laid out as for tsd_accept_joint_trees.  Combined with
  * TSD_SEARCH_LONGEST this is the longest-path search under trajectory drift.
  *

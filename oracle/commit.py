@@ -14,17 +14,25 @@ full, in which case U is empty and no step is taken).
 import numpy as np
 
 
-def commit_accepted(parent, state, accepted_node, unmask_flag, unmask_tok, mask_id, step_base=0):
+def gather_accepted_kv(draft, accepted_node, R):
+    """draft [S, B*R, H, d], accepted_node [S] -> [S, R, H, d]: the draft rows of the accepted node
+    (Appendix A / Section 3.1: the block's K/V under the tokens that were kept)."""
+    draft = np.asarray(draft)
+    return np.stack([draft[s, int(a) * R:(int(a) + 1) * R] for s, a in enumerate(np.asarray(accepted_node))])
+
+
+def commit_accepted(parent, state, accepted_node, unmask_flag, unmask_tok, mask_id, step_base=0, tree_root=0):
     """One sequence.  parent [B], state [B,R] -> dict(root [R] = the next root, fill_step [R] = the
     sequential step at which a row was filled by this pass (-1 for rows it did not fill),
-    step_base = the new step count, n_masked = rows still masked in the next root)."""
+    step_base = the new step count, n_masked = rows still masked in the next root).  tree_root is
+    the index of the tree's root when the arrays hold a forest (Section 3.4: two trees per pass)."""
     parent = np.asarray(parent, dtype=np.int64)
     state = np.asarray(state, dtype=np.int32)
     flag = np.asarray(unmask_flag).astype(bool)
     tok = np.asarray(unmask_tok, dtype=np.int32)
     R = state.shape[1]
     path = [int(accepted_node)]
-    while path[-1] != 0:
+    while path[-1] != tree_root:
         path.append(int(parent[path[-1]]))
     path.reverse()                                   # root .. accepted node
     fill_step = np.full(R, -1, dtype=np.int32)

@@ -233,11 +233,11 @@ int oracle_decode_rule(int R, const int32_t* state, int32_t mask_id,
  *   rule 0 (EXACT): D(c) == U(parent) as sets of (row, token)
  *   rule 1 (TOP1) : every (r, t) in D(c) has t == top1[parent][r]
  *   rule 2 (TOPK) : every (r, t) in D(c) has t among the parent's topk_m most
- *                   probable tokens at r ("fall within top-k")
+ *                   probable tokens at r (the top-k-membership alternative)
  *   rule 3 (PROB) : every (r, t) in D(c) has draft_prob[c][r] > tau, where
  *                   draft_prob[c][r] is the probability the parent's
- *                   distribution at r gives to t ("exceed tau"; strict, as
- *                   in Alg. 1)
+ *                   distribution at r gives to t (the probability-above-tau
+ *                   alternative; strict, as in Alg. 1)
  * Rules 1-3 admit trajectory drift (Section 4, last paragraph); only rule 0
  * is the test of Theorem 1.  top1 holds, per (node, row), the candidate
  * tokens in descending probability, top1_stride apart; entry 0 is the arg-max.
@@ -354,7 +354,7 @@ void oracle_accept(int S, int B, int R, const int32_t* parent,
 
 /* ------------------------------------------------------------------------
  * Probability of every drafted token under its parent's distribution
- * (the quantity the "exceed tau" reading of Section 3.3 tests): for child c,
+ * (the quantity the probability-above-tau reading of Section 3.3 tests): for child c,
  * row r in D(c) with token t,
  *   out[c][r] = exp(z_t - max z) / sum_v exp(z_v - max z),  z = logits[parent(c)][r]
  * (Eq. 2's softmax).  Rows outside D(c), the root, nodes with a parent index

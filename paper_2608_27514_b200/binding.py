@@ -29,6 +29,7 @@ EXPORTS = (
     "tsd_accept_trajectories", "tsd_build_draft_tree",
     "tsd_build_interblock_vis", "tsd_interblock_trigger", "tsd_accept_joint_trees", "tsd_accept_relaxed",
     "tsd_commit_accepted", "tsd_verify_attention_fp8_cache_workspace_bytes", "tsd_verify_attention_fp8_cache",
+    "tsd_gather_accepted_kv", "tsd_selftest_bounded_wait",
 )
 
 
@@ -90,8 +91,11 @@ def lib():
                                              _i32, _i32] + [_vp] * 9
         L.tsd_accept_relaxed.argtypes = ([_i32, _i32, _i32, _i32, _vp, _vp, _i32, _vp, _vp, _i32, _i32, _vp, _i32,
                                           _i64, _i64, _vp, _f32, _i32, _i32] + [_vp] * 10)
-        L.tsd_commit_accepted.argtypes = [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _vp, _vp,
+        L.tsd_commit_accepted.argtypes = [_i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _vp, _vp,
                                           _vp, _vp, _vp, _vp, _vp]
+        L.tsd_gather_accepted_kv.argtypes = [_i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i64, _i64, _i64,
+                                             _vp, _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp]
+        L.tsd_selftest_bounded_wait.argtypes = [_vp, _u32, _vp]
         L.tsd_verify_attention_fp8_cache_workspace_bytes.restype = _sz
         L.tsd_verify_attention_fp8_cache_workspace_bytes.argtypes = [ctypes.POINTER(tsd_layout)]
         L.tsd_verify_attention_fp8_cache.argtypes = (
@@ -295,16 +299,39 @@ def tsd_accept_relaxed(parent, state, n_cur, mask_id, conf, topk_idx, topk_m, lo
 
 def tsd_commit_accepted(parent, state, accepted_node, unmask_flag, unmask_tok, mask_id, tokens=None,
                         block_start=None, root_out=None, fill_step=None, step_base=None, n_masked=None,
-                        status=None, stream=None):
-    """parent [S,B], state [S,B,R]; tokens [S,L] (row stride = tokens.stride(0)); the rest [S] / [S,R]."""
+                        status=None, stream=None, tree_root=0):
+    """parent [S,B], state [S,B,R]; tokens [S,L] (row stride = tokens.stride(0)); the rest [S] / [S,R];
+    tree_root = forest index of the tree's root (the next block's tree of a joint pass)."""
     S, B, R = state.shape
     if tokens is not None:
         assert tokens.dim() == 2 and tokens.stride(1) == 1
     rc = lib().tsd_commit_accepted(
-        S, B, R, _ptr(parent), _ptr(state), _ptr(accepted_node), _ptr(unmask_flag), _ptr(unmask_tok),
+        S, B, R, int(tree_root), _ptr(parent), _ptr(state), _ptr(accepted_node), _ptr(unmask_flag), _ptr(unmask_tok),
         int(mask_id), _ptr(tokens), 0 if tokens is None else tokens.stride(0), _ptr(block_start), _ptr(root_out),
         _ptr(fill_step), _ptr(step_base), _ptr(n_masked), _ptr(status), _stream(stream))
     _check(rc, "tsd_commit_accepted")
+
+
+def tsd_gather_accepted_kv(accepted_node, rows_per_branch, k_draft, v_draft, k_out, v_out, out_row0=None,
+                           status=None, stream=None):
+    """k/v_draft [S, B*R, Hkv, d] -> k/v_out [S, rows, Hkv, d] at row out_row0[s] (views allowed; the
+    last dimension contiguous); v_draft / v_out may both be None."""
+    S, N, H, d = k_draft.shape
+    assert k_draft.stride(3) == 1 and k_out.stride(3) == 1 and k_out.shape[0] == S and k_out.shape[2:] == (H, d)
+    if v_draft is not None:
+        assert v_draft.stride() == k_draft.stride() and v_out.stride() == k_out.stride()
+    rc = lib().tsd_gather_accepted_kv(
+        S, N // rows_per_branch, int(rows_per_branch), H, d, dtype_code(k_draft.dtype), _ptr(accepted_node),
+        _ptr(k_draft), _ptr(v_draft), k_draft.stride(0), k_draft.stride(1), k_draft.stride(2),
+        _ptr(k_out), _ptr(v_out), k_out.stride(0), k_out.stride(1), k_out.stride(2), _ptr(out_row0),
+        k_out.shape[1], _ptr(status), _stream(stream))
+    _check(rc, "tsd_gather_accepted_kv")
+
+
+def tsd_selftest_bounded_wait(status, poll_limit=64, stream=None):
+    """Runs the library's bounded barrier wait on a barrier nothing completes; sets TSD_STATUS_TIMEOUT."""
+    _check(lib().tsd_selftest_bounded_wait(_ptr(status), int(poll_limit), _stream(stream)),
+           "tsd_selftest_bounded_wait")
 
 
 def tsd_verify_attention_fp8_cache_workspace_bytes(layout):

@@ -7,7 +7,7 @@
 // Integer and float compares only: the result is exact.
 //
 // Besides the exact and top-1 tests, the two relaxed readings of the verification test
-// ("fall within top-k / exceed tau"): membership of the drafted token in the parent's first
+// (the top-k-membership and probability-above-tau alternatives of that passage): membership of the drafted token in the parent's first
 // topk_m candidates, and the probability of the drafted token under the parent's distribution,
 // gathered here from the logits and the row's log-sum-exp (one scattered load per drafted token;
 // the vocabulary pass has already produced the log-sum-exp).

@@ -76,7 +76,7 @@ constexpr uint32_t kOffMref = kOffBar + 512;   // exponent offset per row (128 f
 // rotation (3 x 3 x 128 floats each): a softmax warpgroup leaves them for the epilogue and moves on
 constexpr uint32_t kOffLpart = kOffMref + 512;
 constexpr uint32_t kOffMpart = kOffLpart + 3 * 3 * 128 * 4;
-constexpr uint32_t kOffItems = kOffMpart + 3 * 3 * 128 * 4;  // key tiles / cached tiles per item (2 x kMaxItems int32)
+constexpr uint32_t kOffItems = kOffMpart + 3 * 3 * 128 * 4;  // key tiles / cache length per item (2 x kMaxItems int32)
 constexpr uint32_t kSmemBytes = kOffItems + 2 * kMaxItems * 4 + 1024;  // + slack to align the base to 1 KB
 constexpr uint32_t kColO = 0, kColQ = 128, kColS = 256, kColP = 448;  // tensor-memory columns
 constexpr uint32_t kSpinLimit = 1u << 21;
@@ -424,7 +424,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   float* lpart = reinterpret_cast<float*>(base_ptr + kOffLpart);
   float* mpart = reinterpret_cast<float*>(base_ptr + kOffMpart);
   int32_t* item_T = reinterpret_cast<int32_t*>(base_ptr + kOffItems);
-  int32_t* item_nct = item_T + kMaxItems;
+  int32_t* item_clen = item_T + kMaxItems;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -449,7 +449,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int clen = min(max(mask[kHdrWords + s], 0), p.Nc);
     const int n_dt = min(max(mask[p.recs_off + (size_t)(s * p.n_qt + qt) * p.rec_words], 1), p.n_qt);
     const int n_ct = (clen + kKeys - 1) / kKeys;
-    item_nct[it] = n_ct;
+    item_clen[it] = clen;
     item_T[it] = n_ct + 2 * n_dt;
   }
 
@@ -539,7 +539,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         while (is_k && ok && q_issued <= it) issue_q(true);
         int s, h, qt;
         item_coords(it, s, h, qt);
-        const int g = h / p.group, n_ct = item_nct[it], T = item_T[it];
+        const int g = h / p.group, n_ct = (item_clen[it] + kKeys - 1) / kKeys, T = item_T[it];
         const int32_t* rec = mask + p.recs_off + (size_t)(s * p.n_qt + qt) * p.rec_words;
         for (int j = 0; j < T && ok; ++j, ++G) {
           if (is_k) issue_q(false);
@@ -641,6 +641,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       bool ready = false;
       for (int it = 0; it < n_run && ok; ++it) {
         const int T = __shfl_sync(0xffffffffu, item_T[it], 0);
+        const int clen = __shfl_sync(0xffffffffu, item_clen[it], 0);
+        const int n_ct = (clen + kKeys - 1) / kKeys;
+        int s, h, qt;
+        item_coords(it, s, h, qt);
+        const int32_t* rec = mask + p.recs_off + (size_t)(s * p.n_qt + qt) * p.rec_words;
+        const unsigned bits0 = (unsigned)__ldg(rec + 3);  // visibility of the first listed draft tile, asked for early
         // the first P V of an item overwrites O: the epilogue of the previous item must have read it
         if (it > 0) ok = mbar_wait(bar(O_FREE), (it - 1) & 1, abort_flag);
         for (int j = 0; j < T; ++j, ++G) {
@@ -651,6 +657,38 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             ok = ok && mbar_wait(bar(PV_GO + b), (G >> 2) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+          }
+          // A weight of exactly 0 is not enough where V holds Inf or NaN (0 x NaN = NaN): key rows that
+          // no row of the query tile may read are zeroed in shared memory before the MMAs see them.
+          // These are the cached rows past the sequence's cache length (whatever the caller left in the
+          // unused capacity) and the rows of a draft tile's branches that the query tile cannot see.
+          {
+            int z0 = kKeys, z1 = kKeys;  // rows [z0, z1) to zero
+            unsigned dead = 0;           // bit i: rows [32 i, 32 i + 32) to zero (draft tiles)
+            if (j < n_ct) {
+              if (j == n_ct - 1) z0 = clen - j * kKeys;  // 1..64 valid rows
+            } else {
+              const int e = j - n_ct;
+              const unsigned bits = e < 2 ? bits0 : (unsigned)__ldg(rec + 3 + 2 * (e >> 1));  // bit qs*4+ks
+              unsigned seen_slots = 0;
+#pragma unroll
+              for (int qs = 0; qs < 4; ++qs) seen_slots |= (bits >> (4 * qs)) & 15u;
+#pragma unroll
+              for (int w = 0; w < 2; ++w)
+                if (!((seen_slots >> (((e & 1) * kKeys + w * 32) / p.R)) & 1u)) dead |= 1u << w;
+            }
+            if (z0 < z1 || dead) {
+              const uint32_t v_stage = base + kOffV + (uint32_t)b * kKVBytes;
+              if (dead) { z0 = (dead & 1u) ? 0 : 32; z1 = (dead & 2u) ? kKeys : 32; }
+              // 16 chunks of 16 bytes per row (8 per sub-tile): whole rows, so the swizzle does not matter
+              for (int idx = lane; idx < (z1 - z0) * 16; idx += 32) {
+                const int row = z0 + (idx >> 4), ch = idx & 15;
+                const uint32_t a = v_stage + (uint32_t)(ch >> 3) * kSubKV + (uint32_t)row * 128u + (uint32_t)(ch & 7) * 16u;
+                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0u) : "memory");
+              }
+              fence_async_smem();  // the tensor pipe reads shared memory through the async proxy
+              __syncwarp();
+            }
           }
           tc_fence_after();
           if (lane == 0) TSD_TR(7, G);
@@ -706,8 +744,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       int s, h, qt;
       item_coords(it, s, h, qt);
       const int32_t* rec = mask + p.recs_off + (size_t)(s * p.n_qt + qt) * p.rec_words;
-      const int clen = min(max(mask[kHdrWords + s], 0), p.Nc);
-      const int n_ct = item_nct[it], T = item_T[it];
+      const int clen = item_clen[it];
+      const int n_ct = (clen + kKeys - 1) / kKeys, T = item_T[it];
       const int jc = min(4, T - 1);  // the tile at which Q of the next item is copied
       float m_mine = -CUDART_INF_F, l = 0.f;  // the exponent offset this thread used last, its partial row sum
       // tile t goes to warpgroup t mod 3, which is also its S buffer; n_done counts this
@@ -967,6 +1005,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, TSD_STATUS_TIMEOUT);
 }
 
+// The bounded wait of this file on a barrier that nothing ever completes: it gives up after
+// `poll_limit` polls, the block notes it and returns by itself, as a block of the attention kernel
+// does when one of its waits runs out.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint32_t poll_limit) {
+  __shared__ uint64_t bar_mem;
+  __shared__ uint32_t abort_word;
+  const uint32_t b = smem_u32(&bar_mem);
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(b, 0, &abort_word, 0, poll_limit);
+  __syncthreads();
+  if (threadIdx.x == 0 && (!ok || abort_word) && status) atomicOr(status, TSD_STATUS_TIMEOUT);
+}
+
 // ------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1094,3 +1150,12 @@ extern "C" int tsd_attention_trace_read(long long* dst) {
   return (int)cudaMemcpyFromSymbol(dst, tsd::g_attn_trace, sizeof(tsd::g_attn_trace));
 }
 #endif
+
+extern "C" int tsd_selftest_bounded_wait(uint32_t* status, uint32_t poll_limit, tsd_stream_t stream) {
+  if (!status || poll_limit < 1 || poll_limit > (1u << 16)) return TSD_ERR_INVALID_ARG;
+  tsd::bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, poll_limit);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tsd::cuda_fail(e, "bounded_wait_selftest_kernel");
+  return TSD_OK;
+}
+

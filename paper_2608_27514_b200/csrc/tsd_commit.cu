@@ -7,6 +7,7 @@
 // at sequential step step_base + j - 1, the rows of U(accepted node) at step_base + depth.  The
 // next root is written into the sequence's token buffer at the block's position, and the block's
 // step counter moves on by depth + 1 (depth, if the accepted node had nothing left to unmask).
+#include <algorithm>
 #include "tsd_common.cuh"
 
 namespace tsd {
@@ -16,7 +17,7 @@ constexpr int kCommitRowsPerLane = kCommitMaxRows / 32;
 constexpr int kCommitMaxBranches = 256;
 
 __global__ void __launch_bounds__(32)
-commit_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
+commit_kernel(int B, int R, int root, const int32_t* __restrict__ parent, const int32_t* __restrict__ state,
               const int32_t* __restrict__ accepted_node, const uint8_t* __restrict__ unmask_flag,
               const int32_t* __restrict__ unmask_tok, int mask_id, int32_t* __restrict__ tokens,
               int64_t seq_stride, const int32_t* __restrict__ block_start, int32_t* __restrict__ root_out,
@@ -28,19 +29,21 @@ commit_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
   const int32_t* par = parent + (size_t)s * B;
   const int32_t* st = state + (size_t)s * B * R;
   if (lane == 0) {
-    int b = accepted_node ? accepted_node[s] : 0, n = 0;
-    bool bad = b < 0 || b >= B;
-    if (bad) b = 0;
+    // `root` is the forest index of this tree's root (0 for a tree of its own); node and parent
+    // indices are forest indices, and a tree's nodes follow its root
+    int b = accepted_node ? accepted_node[s] : root, n = 0;
+    bool bad = b < root || b >= B;
+    if (bad) b = root;
     s_path[0] = b;
-    while (b > 0 && n < B) {  // parents precede their children, so this ends within B steps
+    while (b > root && n < B) {  // parents precede their children, so this ends within B steps
       const int p = par[b];
-      if (p < 0 || p >= b) { bad = true; break; }
+      if (p < root || p >= b) { bad = true; break; }
       b = p;
       s_path[++n] = b;
     }
     if (bad) {  // inconsistent tree: commit nothing but U(root)
       if (status) atomicOr(status, TSD_STATUS_BAD_PARENT);
-      s_path[0] = 0;
+      s_path[0] = root;
       n = 0;
     }
     s_depth = n;
@@ -64,7 +67,7 @@ commit_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
         v = unmask_tok[(size_t)s * R + r];
         step = base + depth;
       }
-    } else if (st[r] == mask_id) {
+    } else if (st[(size_t)root * R + r] == mask_id) {
       // filled somewhere on the path: by the shallowest node that holds it
       int j = depth;  // s_path[depth - j] is the path node at depth j
       while (j > 1 && st[(size_t)s_path[depth - j + 1] * R + r] != mask_id) --j;
@@ -86,9 +89,70 @@ commit_kernel(int B, int R, const int32_t* __restrict__ parent, const int32_t* _
   }
 }
 
+// The accepted node's draft K/V rows -> a destination of the caller's (one layer per call): 16-byte
+// vectors, one thread each; grid.y = sequence.  The accepted node comes from device memory, so a
+// decode loop can chain this after the acceptance without a read-back.
+__global__ void __launch_bounds__(256)
+gather_accepted_kv_kernel(int B, int R, int H, int vec_per_head, const int32_t* __restrict__ accepted_node,
+                          const uint4* __restrict__ k_src, const uint4* __restrict__ v_src, int64_t ss_b,
+                          int64_t ss_r, int64_t ss_h, uint4* __restrict__ k_dst, uint4* __restrict__ v_dst,
+                          int64_t ds_b, int64_t ds_r, int64_t ds_h, const int32_t* __restrict__ dst_row0,
+                          int dst_rows, uint32_t* __restrict__ status) {
+  const int s = blockIdx.y;
+  const int node = accepted_node ? accepted_node[s] : 0;
+  const int64_t row0 = dst_row0 ? dst_row0[s] : 0;
+  if (node < 0 || node >= B || row0 < 0 || row0 + R > dst_rows) {  // nothing of this sequence is written
+    if (threadIdx.x == 0 && blockIdx.x == 0 && status) atomicOr(status, TSD_STATUS_BAD_INDEX);
+    return;
+  }
+  const int total = R * H * vec_per_head;
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    const int c = t % vec_per_head, h = (t / vec_per_head) % H, r = t / (vec_per_head * H);
+    const int64_t src = s * ss_b + ((int64_t)node * R + r) * ss_r + h * ss_h + c;   // in 16-byte units
+    const int64_t dst = s * ds_b + (row0 + r) * ds_r + h * ds_h + c;
+    k_dst[dst] = k_src[src];
+    if (v_src) v_dst[dst] = v_src[src];
+  }
+}
+
 }  // namespace tsd
 
-extern "C" int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_branch,
+extern "C" int tsd_gather_accepted_kv(int32_t batch, int32_t n_branches, int32_t rows_per_branch, int32_t n_kv_heads,
+                                      int32_t head_dim, int32_t dtype, const int32_t* accepted_node,
+                                      const void* k_draft, const void* v_draft, int64_t d_stride_b,
+                                      int64_t d_stride_row, int64_t d_stride_head, void* k_out, void* v_out,
+                                      int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head,
+                                      const int32_t* out_row0, int32_t out_rows, uint32_t* status,
+                                      tsd_stream_t stream) {
+  if (batch < 0 || n_branches < 1 || n_branches > tsd::kCommitMaxBranches || rows_per_branch < 1 ||
+      rows_per_branch > tsd::kCommitMaxRows || n_kv_heads < 1 || head_dim < 1 || out_rows < rows_per_branch)
+    return TSD_ERR_INVALID_ARG;
+  if (dtype != TSD_F32 && dtype != TSD_BF16) return TSD_ERR_UNSUPPORTED;
+  const int esize = dtype == TSD_F32 ? 4 : 2;
+  if ((head_dim * esize) % 16 != 0) return TSD_ERR_UNSUPPORTED;
+  if (batch == 0) return TSD_OK;
+  if (!k_draft || !k_out || (v_draft == nullptr) != (v_out == nullptr)) return TSD_ERR_INVALID_ARG;
+  const void* ptrs[] = {k_draft, v_draft, k_out, v_out};
+  for (const void* p : ptrs)
+    if (p && !tsd::aligned16(p)) return TSD_ERR_INVALID_ARG;
+  const int64_t strides[] = {d_stride_b, d_stride_row, d_stride_head, o_stride_b, o_stride_row, o_stride_head};
+  for (int64_t st : strides)
+    if (st < 0 || (st * esize) % 16 != 0) return TSD_ERR_INVALID_ARG;
+  if (d_stride_head < head_dim || o_stride_head < head_dim) return TSD_ERR_INVALID_ARG;
+  const int per16 = 16 / esize, vec_per_head = head_dim / per16;
+  const int total = rows_per_branch * n_kv_heads * vec_per_head;
+  dim3 grid((unsigned)std::min((total + 255) / 256, 64), (unsigned)batch);
+  tsd::gather_accepted_kv_kernel<<<grid, 256, 0, stream>>>(
+      n_branches, rows_per_branch, n_kv_heads, vec_per_head, accepted_node, static_cast<const uint4*>(k_draft),
+      static_cast<const uint4*>(v_draft), d_stride_b / per16, d_stride_row / per16, d_stride_head / per16,
+      static_cast<uint4*>(k_out), static_cast<uint4*>(v_out), o_stride_b / per16, o_stride_row / per16,
+      o_stride_head / per16, out_row0, out_rows, status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return tsd::cuda_fail(e, "gather_accepted_kv_kernel");
+  return TSD_OK;
+}
+
+extern "C" int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t rows_per_branch, int32_t tree_root,
                                    const int32_t* parent, const int32_t* state, const int32_t* accepted_node,
                                    const uint8_t* unmask_flag, const int32_t* unmask_tok, int32_t mask_id,
                                    int32_t* tokens, int64_t seq_stride, const int32_t* block_start,
@@ -97,11 +161,12 @@ extern "C" int tsd_commit_accepted(int32_t batch, int32_t n_branches, int32_t ro
   if (batch < 0 || n_branches < 1 || n_branches > tsd::kCommitMaxBranches || rows_per_branch < 1 ||
       rows_per_branch > tsd::kCommitMaxRows)
     return TSD_ERR_INVALID_ARG;
+  if (tree_root < 0 || tree_root >= n_branches) return TSD_ERR_INVALID_ARG;
   if ((unmask_flag == nullptr) != (unmask_tok == nullptr)) return TSD_ERR_INVALID_ARG;
   if (tokens && seq_stride < rows_per_branch) return TSD_ERR_INVALID_ARG;
   if (batch == 0) return TSD_OK;
   if (!parent || !state) return TSD_ERR_INVALID_ARG;
-  tsd::commit_kernel<<<batch, 32, 0, stream>>>(n_branches, rows_per_branch, parent, state, accepted_node,
+  tsd::commit_kernel<<<batch, 32, 0, stream>>>(n_branches, rows_per_branch, tree_root, parent, state, accepted_node,
                                                unmask_flag, unmask_tok, mask_id, tokens, seq_stride, block_start,
                                                root_out, fill_step, step_base, n_masked, status);
   cudaError_t e = cudaGetLastError();

@@ -23,7 +23,6 @@
 #include <limits.h>
 #include <math_constants.h>
 #include <algorithm>
-#include <mutex>
 #include "tsd_common.cuh"
 
 namespace tsd {
@@ -630,25 +629,16 @@ namespace tsd {
 constexpr size_t kStaticScratchBytes = 1u << 20;  // 1 MiB per device
 static __device__ __align__(256) unsigned char g_topk_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-static std::mutex g_scratch_mutex;
-static void* g_scratch_ptr[kMaxDevices] = {};  // device address of g_topk_scratch, per device
-
 // In host code `g_topk_scratch` is only a handle for the runtime, not an address a kernel can use:
-// the device address has to be asked for, once per device, with that device current.
+// the device address has to be asked for, with the device current.  The lookup is a host-side
+// query that allocates nothing; it is repeated on every call rather than remembered, so that the
+// address is never one from before a device reset (the first lookup on a device loads the
+// library's module there, which is why that first call belongs before any stream capture).
 static cudaError_t static_scratch_address(void** out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
+  void* ptr = nullptr;
+  cudaError_t e = cudaGetSymbolAddress(&ptr, g_topk_scratch);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_scratch_mutex);
-  if (!g_scratch_ptr[dev]) {
-    void* ptr = nullptr;
-    e = cudaGetSymbolAddress(&ptr, g_topk_scratch);
-    if (e != cudaSuccess) return e;
-    g_scratch_ptr[dev] = ptr;
-  }
-  *out = g_scratch_ptr[dev];
+  *out = ptr;
   return cudaSuccess;
 }
 
@@ -671,8 +661,10 @@ extern "C" int tsd_confidence_topk_static(const void* logits, int32_t dtype, int
     return TSD_ERR_INVALID_ARG;
   const tsd::TopkPlan p = tsd::topk_plan(n_rows, vocab, k, 16 / esize);
   // this shape would need more scratch than the library carries: the caller has to use
-  // tsd_confidence_topk with a workspace of its own
-  if (p.total_bytes > tsd::kStaticScratchBytes) return TSD_ERR_WORKSPACE;
+  // tsd_confidence_topk with a workspace of its own.  The test is on the documented size
+  // (tsd_confidence_topk_workspace_bytes, the larger of the two dtypes' needs), so that the check a
+  // caller makes beforehand and this one agree.
+  if (tsd_confidence_topk_workspace_bytes(n_rows, vocab, k) > tsd::kStaticScratchBytes) return TSD_ERR_WORKSPACE;
   void* scratch = nullptr;
   if (p.total_bytes > 0) {
     cudaError_t e = tsd::static_scratch_address(&scratch);

@@ -50,8 +50,10 @@ class BlockDecoder:
         t["n"].fill_(1)
         self.fill_step.fill_(-1)
         self.step_base.zero_()
-        self.n_masked.copy_((root_state == self.mask_id).sum(dim=1))
-        self.root.copy_(root_state)
+        # the root alone, nothing accepted, nothing to unmask: the commit kernel copies it to
+        # self.root and counts its masked rows
+        B.tsd_commit_accepted(t["parent"], t["state"], None, None, None, self.mask_id, root_out=self.root,
+                              n_masked=self.n_masked, status=self.step.status)
         self.n_forward = 0
 
     def advance(self, logits, tokens=None, block_start=None):

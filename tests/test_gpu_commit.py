@@ -159,3 +159,98 @@ def test_theorem1_on_the_device(tau, search):
     assert np.array_equal(seq[2], spec[2])             # same number of sequential steps
     assert seq[3] == seq[2].max()                      # without drafts: one forward per step
     assert spec[3] < seq[3]                            # speculation saved forwards
+
+
+def test_commit_both_trees_of_a_joint_pass():
+    # Section 3.4: one pass carries the tree of the current block (root 0) and a tree of the next
+    # block (root n_cur); parents and accepted nodes are forest indices.  Each tree commits on its own.
+    rng = np.random.default_rng(21)
+    S, R, V, n_cur, n_nxt = 9, 32, 500, 7, 5
+    Bn, M = n_cur + n_nxt, 500
+    pa, sa, acc_a, fa, ta, _ = _valid_trees(rng, S, n_cur, R, V)
+    pb, sb, acc_b, fb, tb, _ = _valid_trees(rng, S, n_nxt, R, V)
+    parent = np.concatenate([pa, np.where(pb < 0, -1, pb + n_cur)], axis=1).astype(np.int32)
+    state = np.concatenate([sa, sb], axis=1)
+    for root_idx, acc, flag, tok in ((0, acc_a, fa, ta), (n_cur, acc_b + n_cur, fb, tb)):
+        root = torch.empty((S, R), dtype=torch.int32, device=DEV)
+        fill = torch.full((S, R), -1, dtype=torch.int32, device=DEV)
+        base, n_masked = torch.full((S,), 3, dtype=torch.int32, device=DEV), torch.empty(S, dtype=torch.int32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.tsd_commit_accepted(_t(parent, torch.int32), _t(state, torch.int32), _t(acc, torch.int32),
+                              _t(flag, torch.uint8), _t(tok, torch.int32), M, root_out=root, fill_step=fill,
+                              step_base=base, n_masked=n_masked, status=status, tree_root=root_idx)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for s in range(S):
+            o = C.commit_accepted(parent[s], state[s], acc[s], flag[s], tok[s], M, 3, tree_root=root_idx)
+            assert np.array_equal(root[s].cpu().numpy(), o["root"])
+            assert np.array_equal(fill[s].cpu().numpy(), o["fill_step"])
+            assert int(base[s]) == o["step_base"] and int(n_masked[s]) == o["n_masked"]
+    # an accepted node of the other tree is outside this one: reported, U(root) only
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    root = torch.empty((S, R), dtype=torch.int32, device=DEV)
+    B.tsd_commit_accepted(_t(parent, torch.int32), _t(state, torch.int32), _t(acc_a, torch.int32), None, None, M,
+                          root_out=root, status=status, tree_root=n_cur)
+    torch.cuda.synchronize()
+    assert B.tsd_check_status(status) == B.TSD_ERR_DEVICE_DATA
+    assert np.array_equal(root.cpu().numpy(), state[:, n_cur])
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_gather_accepted_kv_matches_oracle(dtype):
+    # the accepted node's draft K/V rows -> a slot of the caller's cache, from strided views of a
+    # fused projection output into a strided view of a wider cache tensor
+    g = torch.Generator(device=DEV).manual_seed(3)
+    S, Bn, R, H, d, rows = 5, 6, 32, 3, 128, 200
+    qkv = torch.randn((S, Bn * R, 2 * H + 1, d), generator=g, device=DEV).to(dtype)
+    k_draft, v_draft = qkv[:, :, 1:1 + H], qkv[:, :, 1 + H:]
+    cache = torch.full((S, rows, 2 * H, d), 7.0, dtype=dtype, device=DEV)
+    k_out, v_out = cache[:, :, :H], cache[:, :, H:]
+    acc = torch.tensor([3, 0, 5, 1, 2], dtype=torch.int32, device=DEV)
+    row0 = torch.tensor([0, 168, 10, 64, 96], dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.tsd_gather_accepted_kv(acc, R, k_draft, v_draft, k_out, v_out, row0, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    wk = C.gather_accepted_kv(k_draft.float().cpu().numpy(), acc.cpu().numpy(), R)
+    wv = C.gather_accepted_kv(v_draft.float().cpu().numpy(), acc.cpu().numpy(), R)
+    want = np.full((S, rows, 2 * H, d), 7.0, np.float32)
+    for s in range(S):
+        r0 = int(row0[s])
+        want[s, r0:r0 + R, :H] = wk[s]
+        want[s, r0:r0 + R, H:] = wv[s]
+    assert np.array_equal(cache.float().cpu().numpy(), want)       # a copy: bit-exact, nothing else touched
+    # K only, default node (0) and default destination row (0)
+    cache.fill_(7.0)
+    B.tsd_gather_accepted_kv(None, R, k_draft, None, k_out, None)
+    torch.cuda.synchronize()
+    assert torch.equal(k_out[:, :R], k_draft[:, :R]) and (cache[:, R:] == 7.0).all() and (v_out == 7.0).all()
+    # a node outside the tree, a destination past the end: reported, those sequences untouched
+    cache.fill_(7.0)
+    bad_acc = torch.tensor([3, 6, 5, -1, 2], dtype=torch.int32, device=DEV)
+    bad_row0 = torch.tensor([0, 0, 169, 0, 96], dtype=torch.int32, device=DEV)
+    B.tsd_gather_accepted_kv(bad_acc, R, k_draft, v_draft, k_out, v_out, bad_row0, status)
+    torch.cuda.synchronize()
+    assert B.tsd_check_status(status) == B.TSD_ERR_DEVICE_DATA
+    assert (cache[1] == 7.0).all() and (cache[2] == 7.0).all() and (cache[3] == 7.0).all()
+    assert torch.equal(k_out[0, :R], k_draft[0, 3 * R:4 * R]) and torch.equal(v_out[4, 96:96 + R], v_draft[4, 2 * R:3 * R])
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    # the library's bounded barrier wait on a barrier nothing completes: the kernel gives up after
+    # the poll limit, returns by itself and raises the time-out bit; the device keeps working
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.tsd_selftest_bounded_wait(status, poll_limit=32)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1
+    assert B.tsd_check_status(status) == B.TSD_ERR_TIMEOUT
+    x = torch.arange(1000, device=DEV).sum().item()                # the context still answers
+    assert x == 499500
+    # the attention stage reports through the same word: a clean run leaves it at 0
+    from paper_2608_27514_b200 import workloads as W
+    cfg = W.small(W.CONFIGS["cfg2"], B=4, Nc=64, Hq=2, Hkv=2)
+    step = VerifyStep.for_config(cfg, DEV)
+    attn = W.attention_inputs(cfg, DEV)
+    step.attention(attn["q"], attn["k_cache"], attn["v_cache"], attn["k_draft"], attn["v_draft"], attn["sm_scale"])
+    torch.cuda.synchronize()
+    assert B.tsd_check_status(step.status) == B.TSD_OK

@@ -203,6 +203,39 @@ def test_attention_poisoned_branches_do_not_leak(flags):
 
 
 @pytest.mark.parametrize("flags", PATHS)
+def test_attention_unreadable_rows_may_hold_anything(flags):
+    # Inf / NaN in rows that no query row of a tile may read must not reach its output (a weight of
+    # 0 times NaN is NaN): cached rows past cache_lens, whatever the unused capacity holds, and
+    # the rows of the branches of a listed draft tile that the query tile cannot see.
+    cfg = W.small(W.CONFIGS["cfg2"], S=2, B=8, R=32, Nc=200, Hq=2, Hkv=1)
+    attn = W.attention_inputs(cfg, DEV)
+    lens = torch.tensor([137, 64], dtype=torch.int32, device=DEV)
+    for s_, n in enumerate(lens.tolist()):
+        attn["k_cache"][s_, n:] = float("nan")
+        attn["v_cache"][s_, n:] = float("inf")
+        attn["v_cache"][s_, n::2] = float("nan")
+    # query tile 0 (branches 0-3) lists draft tile 1 only because branch 0 reads branch 4: the
+    # rows of branches 5-7 are loaded with it and are unreadable for every row of the tile
+    vis = np.zeros((cfg.S, cfg.B, 1), dtype=np.int64)
+    vis[:, 0, 0] = 1 << 4
+    bad = slice(5 * cfg.R, 8 * cfg.R)
+    attn["k_draft"][:, bad] = float("nan")
+    attn["v_draft"][:, bad] = float("-inf")
+    vis_t = torch.from_numpy(vis).to(DEV)
+    step, _ = _run_attention(cfg, attn, flags, vis_t, lens)
+    mask = oracle.dense_mask(cfg.S, cfg.B, cfg.R, cfg.Nc, vis.astype(np.uint64), lens.cpu().numpy())
+    # branches 5-7 read their own NaN, and branch 4 shares its query tile with them (draft rows
+    # that some row of a query tile may read have to be finite): unspecified
+    good = slice(0, 4 * cfg.R)
+    ref, ref_lse = oracle.masked_attention(_np(attn["q"]), _np(attn["k_cache"]), _np(attn["v_cache"]),
+                                           _np(attn["k_draft"]), _np(attn["v_draft"]), mask, attn["sm_scale"])
+    got = _np(step.out).astype(np.float64)[:, good]
+    assert np.isfinite(got).all()
+    assert (np.abs(got - ref[:, good]) <= _attn_tol(cfg, ref[:, good])).all()
+    assert np.abs(step.attn_lse.cpu().numpy()[:, :, good] - ref_lse[:, :, good]).max() <= 2e-2
+
+
+@pytest.mark.parametrize("flags", PATHS)
 def test_attention_sharp_scores(flags):
     # queries scaled x4: near one-hot softmax rows, where a leaked or dropped key would show
     cfg = W.small(W.CONFIGS["cfg2"], B=8, Nc=512, Hq=2, Hkv=2)

@@ -1,4 +1,4 @@
-"""GPU parity of the relaxed acceptance tests (Section 3.3: "fall within top-k / exceed tau") against
+"""GPU parity of the relaxed acceptance tests (Section 3.3: the top-k-membership and probability-above-tau alternatives) against
 the oracle: hand-worked trees, random trees scored from full logits through the vocabulary pass,
 strictness of the probability test, and the two-tree form."""
 import numpy as np

@@ -32,6 +32,28 @@ def test_hand_worked_pass():
     assert o["root"].tolist() == [2, 1] and o["fill_step"].tolist() == [0, -1] and o["step_base"] == 1
 
 
+def test_hand_worked_forest_and_kv_hand_over():
+    # Two trees in one pass (Section 3.4): nodes 0-2 belong to the current block (root 0), nodes 3-5
+    # to the next block (root 3); parents are forest indices.  R = 3, mask = 9.
+    M = 9
+    parent = [-1, 0, 1, -1, 3, 3]
+    state = [[M, M, 1], [2, M, 1], [2, 3, 1],      # chain 0 -> 1 -> 2
+             [M, M, M], [4, M, M], [M, 5, M]]      # root 3 with children 4 and 5
+    # next block's tree: node 4 accepted (depth 1), U(node 4) = row 2 with token 7
+    o = C.commit_accepted(parent, state, 4, [0, 0, 1], [-1, -1, 7], M, step_base=2, tree_root=3)
+    assert o["root"].tolist() == [4, M, 7] and o["fill_step"].tolist() == [2, -1, 3]
+    assert o["step_base"] == 4 and o["n_masked"] == 1
+    # current block's tree: node 2 accepted (depth 2), already full
+    o = C.commit_accepted(parent, state, 2, [0, 0, 0], [-1, -1, -1], M, step_base=0, tree_root=0)
+    assert o["root"].tolist() == [2, 3, 1] and o["fill_step"].tolist() == [0, 1, -1] and o["step_base"] == 2
+    # K/V hand-over: 2 sequences, 3 nodes of R = 2 rows, 1 head, d = 2; value = 100 s + 10 row + c
+    draft = np.array([[[[100 * s + 10 * i + c for c in range(2)]] for i in range(6)] for s in range(2)], np.float32)
+    got = C.gather_accepted_kv(draft, [2, 0], 2)
+    assert got.shape == (2, 2, 1, 2)
+    assert got[0].reshape(-1).tolist() == [40, 41, 50, 51]          # node 2 of sequence 0: rows 4, 5
+    assert got[1].reshape(-1).tolist() == [100, 101, 110, 111]      # node 0 of sequence 1: rows 0, 1
+
+
 @pytest.mark.parametrize("tau", [0.9, 1.5])
 @pytest.mark.parametrize("mode", ["peek", "alg1", "heuristic"])
 def test_committed_steps_are_the_sequential_steps(tau, mode):

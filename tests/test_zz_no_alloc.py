@@ -8,9 +8,11 @@ call cudaMalloc).  The test uses few rows so that rows are split into segments, 
 that needs scratch at all."""
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_27514_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -40,21 +42,35 @@ def _static(x, k):
     return out
 
 
+def _check_against_oracle(x, k, got):
+    host = x.float().cpu().numpy() if x.dtype == torch.bfloat16 else x.cpu().numpy()
+    r_conf, r_idx, r_prob, r_lse = oracle.confidence_topk(host, k)
+    assert np.array_equal(got[1].cpu().numpy(), r_idx)                       # indices: bit-exact
+    assert np.abs(got[0].cpu().numpy() - r_conf).max() <= 1e-5
+    assert np.abs(got[2].cpu().numpy() - r_prob).max() <= 1e-5
+    assert np.abs(got[3].cpu().numpy() - r_lse).max() <= 1e-4
+
+
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
     g = torch.Generator(device=DEV).manual_seed(77)
     k = 3
-    # two different inputs back to back: the second call finds the first call's leftovers in the
-    # shared array and must not be affected by them
+    # different inputs back to back: each call finds the previous call's leftovers in the shared
+    # array and must not be affected by them.  The shapes differ in segments per row and in k, so
+    # that the partial-result slots of one call overlap the ticket words of another, and both
+    # element types take part.
     xa = (torch.randn((100, 126464), generator=g, device=DEV) * 3).bfloat16()
     xb = (torch.randn((40, 50000), generator=g, device=DEV) * 3).bfloat16()
+    xc = torch.randn((7, 90000), generator=g, device=DEV) * 3                  # fp32
+    xd = (torch.randn((3, 300000), generator=g, device=DEV) * 3).bfloat16()
     assert 0 < B.tsd_confidence_topk_workspace_bytes(100, 126464, k) <= B.tsd_confidence_topk_static_capacity()
-    for x in (xa, xb, xa):
-        ref = _regular(x, k)
-        got = _static(x, k)
+    for x, kk in ((xa, k), (xb, k), (xc, 8), (xa, k), (xd, 1), (xc, 2)):
+        ref = _regular(x, kk)
+        got = _static(x, kk)
         assert torch.equal(got[1], ref[1])                         # indices: bit-exact
         for a, b in ((got[0], ref[0]), (got[2], ref[2])):          # probabilities: the suite's 1e-5
             assert (a - b).abs().max().item() <= 1e-5
         assert (got[3] - ref[3]).abs().max().item() <= 1e-4
+        _check_against_oracle(x, kk, got)                          # and the definition itself
 
 
 def test_static_scratch_rejects_what_does_not_fit():
