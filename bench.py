@@ -63,11 +63,22 @@ def algorithmic(cfg):
     return dict(attn_flops=attn_flops, attn_bytes=attn_bytes, topk_bytes=topk_bytes)
 
 
+def input_copies(cfg):
+    """How many copies of the inputs the timed loops rotate through, so that L2 cannot hold them."""
+    alg = algorithmic(cfg)
+    in_bytes = alg["attn_bytes"] + alg["topk_bytes"]
+    return (1 if in_bytes > 2 * L2_BYTES else int(-(-ROTATE_BYTES // in_bytes))), in_bytes
+
+
 def base_config(cfg, world=1):
-    """The workload description both arms report."""
+    """The workload description: identical for both arms."""
+    n_copies, in_bytes = input_copies(cfg)
     return dict(workload=cfg.name, batch=cfg.S, branches=cfg.B, rows_per_branch=cfg.R, rows=cfg.rows,
                 n_cache=cfg.Nc, q_heads=cfg.Hq, kv_heads=cfg.Hkv, head_dim=cfg.d, vocab=cfg.V, k=cfg.k,
-                tau=cfg.tau, attention_layers_per_step=1, parallelism="replicas" if world > 1 else "1gpu")
+                tau=cfg.tau, attention_layers_per_step=1, parallelism="replicas" if world > 1 else "1gpu",
+                l2_hygiene=("inputs larger than L2" if n_copies == 1 else
+                            "rotating %d input copies (%.0f MB total, L2 is 126 MB)"
+                            % (n_copies, n_copies * in_bytes / 1e6)))
 
 
 class ClockSampler:
@@ -112,6 +123,17 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def time_oracle_sample(cfg, attn, vi, budget_s, oracle, np):
     """Times the oracle on a bounded sample and extrapolates to the full workload.
 
@@ -144,23 +166,35 @@ def time_oracle_sample(cfg, attn, vi, budget_s, oracle, np):
     t_k1, _ = topk_sample(min(cfg.rows, 4 * threads))
     per_head = t_a1
     per_row = t_k1 / min(cfg.rows, 4 * threads)
-    n_kv = max(1, min(cfg.Hkv, int(0.5 * budget_s / max(per_head, 1e-6))))
-    n_rows = max(1, min(cfg.rows, int(0.5 * budget_s / max(per_row, 1e-9))))
-    t_attn = attn_sample(n_kv)
-    t_topk, (conf, idx, prob, _) = topk_sample(n_rows)
+    # the timed part is repeated and the median taken: a single sub-second sample moved by 40 %
+    # from run to run
+    # 5 repeats of a sample that fills the budget; where the whole workload costs less than that,
+    # more repeats of the whole workload (up to 101)
+    whole = per_head * cfg.Hkv + per_row * cfg.rows
+    repeats = int(max(5, min(101, budget_s / max(whole, 1e-6)))) | 1
+    n_kv = max(1, min(cfg.Hkv, int(0.5 * budget_s / repeats / max(per_head, 1e-6))))
+    n_rows = max(1, min(cfg.rows, int(0.5 * budget_s / repeats / max(per_row, 1e-9))))
+    t_attn = statistics.median(attn_sample(n_kv) for _ in range(repeats))
+    topk_runs = [topk_sample(n_rows) for _ in range(repeats)]
+    t_topk = statistics.median(t for t, _ in topk_runs)
+    conf, idx, prob, _ = topk_runs[-1][1]
     # acceptance in full, on confidences of the right shape (values do not change its cost)
     conf_full = np.resize(conf.astype(np.float32), cfg.rows).reshape(S, B, R)
     top1_full = np.resize(idx[:, 0], cfg.rows).reshape(S, B, R)
-    t0 = time.perf_counter()
-    oracle.accept(vi["parent"].cpu().numpy(), vi["state"].cpu().numpy(), vi["mask_id"], conf_full,
-                  top1_full, cfg.tau)
-    t_acc = time.perf_counter() - t0
+    acc_runs = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.accept(vi["parent"].cpu().numpy(), vi["state"].cpu().numpy(), vi["mask_id"], conf_full,
+                      top1_full, cfg.tau)
+        acc_runs.append(time.perf_counter() - t0)
+    t_acc = statistics.median(acc_runs)
     t_full = t_attn * (cfg.Hkv / n_kv) * S + t_topk * (cfg.rows / n_rows) + t_acc
     sample = ("attention: sequence 0, %d of %d kv heads (%d query heads), all %d rows; top-k: first %d of "
-              "%d rows; acceptance: all %d sequences; scaled to the full step"
-              % (n_kv, cfg.Hkv, n_kv * group, cfg.N, n_rows, cfg.rows, S))
+              "%d rows; acceptance: all %d sequences; median of %d repeats each; scaled to the full step"
+              % (n_kv, cfg.Hkv, n_kv * group, cfg.N, n_rows, cfg.rows, S, repeats))
     return dict(value=cfg.rows / t_full, unit=UNIT, cores=threads, kind="oracle", sample=sample,
-                seconds_timed=t_attn + t_topk + t_acc,
+                cpu_model=cpu_model(), build=oracle.BUILD_FLAGS,
+                seconds_timed=repeats * (t_attn + t_topk + t_acc),
                 stage_seconds_full=dict(attention=t_attn * (cfg.Hkv / n_kv) * S,
                                         topk=t_topk * (cfg.rows / n_rows), accept=t_acc))
 
@@ -191,51 +225,20 @@ def run_reference(args, cfg):
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
-                config=dict(base_config(cfg), note="CPU oracle, fp64, bounded sample scaled to the full step"),
+                config=base_config(cfg), note="CPU oracle, fp64, bounded sample scaled to the full step",
                 cpu_baseline=dict(value=value, unit=UNIT, cores=last["cores"], kind="oracle",
-                                  sample=last["sample"]),
+                                  sample=last["sample"], cpu_model=last["cpu_model"], build=last["build"]),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--impl", default="tsd", choices=["tsd", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graph replay")
-    ap.add_argument("--graph-per-step", action="store_true", help="one graph launch per step instead of one per round of input copies")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "tsd" else args.warmup
-
-    from paper_2608_27514_b200 import workloads as W
-    cfg = W.CONFIGS[args.workload]
-    if args.impl == "reference":
-        run_reference(args, cfg)
-        return
-
-    import numpy as np
-    import torch
-    from paper_2608_27514_b200 import binding as B
-    from paper_2608_27514_b200.step import VerifyStep
-
-    from paper_2608_27514_b200 import replicas
-    rank, local_rank, world = replicas.world()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    B.lib()  # fail loudly if the CUDA library is missing
-    torch.cuda.set_device(local_rank)
-    dev = "cuda:%d" % local_rank
-    replicas.init("nccl", dev)
-
+def measure_workload(cfg, args, torch, np, B, W, VerifyStep, replicas, dev, local_rank, world, pk, full):
+    """One workload: region A (K whole steps by CUDA graph replay), region B (each stage alone) and,
+    when `full`, the end-to-end loop and the stages that are timed for context only.  Returns the
+    figures as a dict; every tensor it made is dropped on return."""
     alg = algorithmic(cfg)
-    pk = peaks()
-    in_bytes = alg["attn_bytes"] + alg["topk_bytes"]
-    n_copies = 1 if in_bytes > 2 * L2_BYTES else int(np.ceil(ROTATE_BYTES / in_bytes))
+    n_copies, in_bytes = input_copies(cfg)
     sets = []
     base_attn = W.attention_inputs(cfg, dev)
     base_vi = W.verify_inputs(cfg, dev)
@@ -248,6 +251,7 @@ def main():
         sets.append((step, attn, vi))
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
+    steps = args.steps if full else max(3, min(args.steps, 20))
 
     def run_step(i):
         step, attn, vi = sets[i % n_copies]
@@ -307,7 +311,7 @@ def main():
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    do_steps(first, args.steps)
+    do_steps(first, steps)
     e1.record(stream)
     barrier()
     elapsed_ms = e0.elapsed_time(e1)
@@ -316,7 +320,7 @@ def main():
 
     # ---------------- timed region B: each stage alone, back-to-back launches on rotating inputs,
     # replayed from a CUDA graph so that the host's launch cost does not set the pace
-    def time_stage(fn, min_seconds=0.25):
+    def stage_graph(fn):
         g = torch.cuda.CUDAGraph()
         per_graph = max(n_copies, 4)
         fn(0)
@@ -327,6 +331,12 @@ def main():
         for _ in range(3):
             g.replay()
         torch.cuda.synchronize()
+        return g, per_graph
+
+    def time_stage(fn, min_seconds=0.25):
+        """Sustained: the stage back to back for at least min_seconds (a tensor-bound stage runs
+        into the power cap and its lower clocks, as it would inside a long job)."""
+        g, per_graph = stage_graph(fn)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         g.replay()
@@ -340,6 +350,30 @@ def main():
         b.record(stream)
         torch.cuda.synchronize()
         return a.elapsed_time(b) * 1e-3 / (reps * per_graph)
+
+    def time_stage_burst(fn, bursts=5, burst_seconds=0.01, idle_seconds=0.25):
+        """Burst: the best of a few short runs, each after an idle pause, which is how the tensor
+        peak this is compared with was taken (best of ten single GEMMs)."""
+        g, per_graph = stage_graph(fn)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        once = max(a.elapsed_time(b) * 1e-3, 1e-6)
+        reps = int(min(max(burst_seconds / once, 2), 2000))
+        best = None
+        for _ in range(bursts):
+            time.sleep(idle_seconds)
+            g.replay()                       # clocks and caches up, not counted
+            a.record(stream)
+            for _ in range(reps):
+                g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            t = a.elapsed_time(b) * 1e-3 / (reps * per_graph)
+            best = t if best is None else min(best, t)
+        return best
 
     def f_attn(i):
         step, attn, vi = sets[i % n_copies]
@@ -378,7 +412,7 @@ def main():
     # branches span two blocks: same batch, heads and cache, one block of 32 rows per branch, the
     # last 4 branches = a W1D3 tree of the next block, joint visibility from the library
     ib = None
-    if cfg.R == 64 and cfg.B > 4:
+    if full and cfg.R == 64 and cfg.B > 4:
         ib_cfg = W.small(cfg, R=32)
         ib_attn = W.attention_inputs(ib_cfg, dev)
         ib_step = VerifyStep.for_config(ib_cfg, dev)
@@ -394,7 +428,7 @@ def main():
     # the 8-bit K/V cache variant (no counterpart in the paper): the caches of every input copy as
     # e4m3 codes with one scale per (sequence, kv head); timed for context, not part of the step
     fp8_sets = []
-    if cfg.dtype == "bf16" and cfg.Nc > 0:
+    if full and cfg.dtype == "bf16" and cfg.Nc > 0:
         fp8_ws = torch.empty(max(B.tsd_verify_attention_fp8_cache_workspace_bytes(sets[0][0].layout), 16),
                              dtype=torch.uint8, device=dev)
         for step_c, attn_c, _ in sets:
@@ -415,9 +449,11 @@ def main():
 
     # the tensor-heavy stage last: it drives the GPU into its power cap, which would lower the
     # clocks the other two are measured at
-    t_tree = time_stage(f_tree, 0.05)
-    t_acc_prob = time_stage(f_acc_prob, 0.05)
-    t_acc, t_topk, t_attn = time_stage(f_acc, 0.05), time_stage(f_topk), time_stage(f_attn)
+    t_tree = time_stage(f_tree, 0.05) if full else None
+    t_acc_prob = time_stage(f_acc_prob, 0.05) if full else None
+    t_acc, t_topk = time_stage(f_acc, 0.05), time_stage(f_topk)
+    t_attn_burst = time_stage_burst(f_attn)
+    t_attn = time_stage(f_attn)
     if ib is not None:
         ib["seconds"] = time_stage(f_ib)
         ib_step.check_status()
@@ -425,67 +461,82 @@ def main():
     clocks = sampler.stop()
 
     # ---------------- end to end: pinned host inputs -> device -> step -> host results
-    step0, attn0, vi0 = sets[0]
-    h_names = ["q", "k_draft", "v_draft"]
-    host = {k: attn0[k].cpu().pin_memory() for k in h_names}
-    host_logits = vi0["logits"].cpu().pin_memory()
-    host_parent, host_state = vi0["parent"].cpu().pin_memory(), vi0["state"].cpu().pin_memory()
-    res_names = ["accepted_node", "accepted_len", "n_new_tokens", "unmask_flag", "unmask_tok"]
-    host_out = {k: torch.empty_like(getattr(step0, k), device="cpu").pin_memory() for k in res_names}
-    h2d = sum(t.numel() * t.element_size() for t in list(host.values()) + [host_logits, host_parent, host_state])
-    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+    e2e = None
+    if full:
+        step0, attn0, vi0 = sets[0]
+        h_names = ["q", "k_draft", "v_draft"]
+        host = {k: attn0[k].cpu().pin_memory() for k in h_names}
+        host_logits = vi0["logits"].cpu().pin_memory()
+        host_parent, host_state = vi0["parent"].cpu().pin_memory(), vi0["state"].cpu().pin_memory()
+        res_names = ["accepted_node", "accepted_len", "n_new_tokens", "unmask_flag", "unmask_tok"]
+        host_out = {k: torch.empty_like(getattr(step0, k), device="cpu").pin_memory() for k in res_names}
+        h2d = sum(t.numel() * t.element_size() for t in list(host.values()) + [host_logits, host_parent, host_state])
+        d2h = sum(t.numel() * t.element_size() for t in host_out.values())
 
-    def e2e_step():
-        for k in h_names:
-            attn0[k].copy_(host[k], non_blocking=True)
-        vi0["logits"].copy_(host_logits, non_blocking=True)
-        vi0["parent"].copy_(host_parent, non_blocking=True)
-        vi0["state"].copy_(host_state, non_blocking=True)
-        step0.run(attn0, vi0["logits"], vi0["parent"], vi0["state"], vi0["mask_id"], cfg.tau)
-        for k in res_names:
-            host_out[k].copy_(getattr(step0, k), non_blocking=True)
-        stream.synchronize()   # the caller needs the accepted node before planning the next step
+        def e2e_step():
+            for k in h_names:
+                attn0[k].copy_(host[k], non_blocking=True)
+            vi0["logits"].copy_(host_logits, non_blocking=True)
+            vi0["parent"].copy_(host_parent, non_blocking=True)
+            vi0["state"].copy_(host_state, non_blocking=True)
+            step0.run(attn0, vi0["logits"], vi0["parent"], vi0["state"], vi0["mask_id"], cfg.tau)
+            for k in res_names:
+                host_out[k].copy_(getattr(step0, k), non_blocking=True)
+            stream.synchronize()   # the caller needs the accepted node before planning the next step
 
-    e2e_steps = max(3, min(args.steps, 20))
-    for _ in range(2):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    b.record(stream)
-    barrier()
-    e2e_ms = max(a.elapsed_time(b), (time.perf_counter() - t0) * 1e3) / e2e_steps
+        e2e_steps = max(3, min(args.steps, 20))
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e_ms = max(a.elapsed_time(b), (time.perf_counter() - t0) * 1e3) / e2e_steps
+        e2e = dict(ms=e2e_ms, h2d=int(h2d), d2h=int(d2h))
 
     # ---------------- reduce over ranks (replicas: the slowest rank sets the time)
-    elapsed_ms, e2e_ms = replicas.max_over_ranks([elapsed_ms, e2e_ms], dev)
-    ms_per_step = elapsed_ms / args.steps
+    if e2e is not None:
+        elapsed_ms, e2e["ms"] = replicas.max_over_ranks([elapsed_ms, e2e["ms"]], dev)
+    else:
+        elapsed_ms = replicas.max_over_ranks([elapsed_ms], dev)[0]
+    ms_per_step = elapsed_ms / steps
     value = world * cfg.rows / (ms_per_step * 1e-3)
 
-    # ---------------- roofline of the dominant kernel (+ every stage, for context)
+    # ---------------- roofline of every stage
     attn_flop_time = alg["attn_flops"] / (pk["tflops"] * 1e12)
     attn_byte_time = alg["attn_bytes"] / (pk["hbm_gbs"] * 1e9)
     attn_bound = "tensor" if attn_flop_time >= attn_byte_time else "hbm"
+    roof_s = max(attn_flop_time, attn_byte_time)
     stages = dict(
-        attention=dict(seconds=t_attn, bound=attn_bound, roofline_seconds=max(attn_flop_time, attn_byte_time),
-                       frac=max(attn_flop_time, attn_byte_time) / t_attn,
-                       tflops=alg["attn_flops"] / t_attn / 1e12, gbs=alg["attn_bytes"] / t_attn / 1e9,
-                       # the stage loop runs for a quarter of a second under the power cap: the fraction
-                       # of the sustained cuBLAS figure is given beside the (conservative) burst one
-                       frac_of_sustained_tensor_peak=alg["attn_flops"] / t_attn / 1e12 / pk["tflops_sustained"]),
+        attention=dict(
+            # `seconds` is the sustained figure (the stage back to back for a quarter of a second:
+            # a tensor-bound stage then runs under the power cap at lower clocks); `seconds_burst`
+            # is the best of a few 10 ms runs after idle pauses, the conditions under which the
+            # burst tensor peak was measured.  Each time is set against the peak taken the same way.
+            seconds=t_attn, seconds_burst=t_attn_burst, bound=attn_bound, roofline_seconds=roof_s,
+            frac=roof_s / t_attn, frac_burst=roof_s / t_attn_burst,
+            tflops=alg["attn_flops"] / t_attn / 1e12, tflops_burst=alg["attn_flops"] / t_attn_burst / 1e12,
+            gbs=alg["attn_bytes"] / t_attn / 1e9,
+            frac_of_sustained_tensor_peak=alg["attn_flops"] / t_attn / 1e12 / pk["tflops_sustained"],
+            algorithmic_flops=alg["attn_flops"], algorithmic_bytes=alg["attn_bytes"]),
         topk=dict(seconds=t_topk, bound="hbm", roofline_seconds=alg["topk_bytes"] / (pk["hbm_gbs"] * 1e9),
-                  frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9),
+                  frac=alg["topk_bytes"] / t_topk / (pk["hbm_gbs"] * 1e9), gbs=alg["topk_bytes"] / t_topk / 1e9,
+                  algorithmic_bytes=alg["topk_bytes"]),
         accept=dict(seconds=t_acc),
-        accept_relaxed_prob_longest=dict(seconds=t_acc_prob, note="Section 3.3's probability-above-tau reading with the "
-                                         "gather of the drafted tokens' probabilities; not part of the step"),
-        tree_build_next_step=dict(seconds=t_tree, note="Alg. 1 tree construction (W3 D3) for the next step; not part of the step"),
     )
+    if full:
+        stages["accept_relaxed_prob_longest"] = dict(
+            seconds=t_acc_prob, note="Section 3.3's probability-above-tau reading with the "
+            "gather of the drafted tokens' probabilities; not part of the step")
+        stages["tree_build_next_step"] = dict(
+            seconds=t_tree, note="Alg. 1 tree construction (W3 D3) for the next step; not part of the step")
     if t_fp8 is not None:
         stages["attention_fp8_cache"] = dict(
-            seconds=t_fp8, note="e4m3 K/V cache expanded into a scratch buffer, then the same attention; the cache "
-            "itself takes %.1f MB instead of %.1f MB; not part of the step"
+            seconds=t_fp8, note="e4m3 K/V cache; the cache itself takes %.1f MB instead of %.1f MB; not part of the step"
             % (2 * cfg.S * cfg.Nc * cfg.Hkv * cfg.d / 1e6, 4 * cfg.S * cfg.Nc * cfg.Hkv * cfg.d / 1e6))
     if ib is not None:
         stages["attention_interblock_paper_form"] = dict(
@@ -500,47 +551,105 @@ def main():
                     algorithmic_bytes=alg["topk_bytes"], peak_source=pk["source"])
     elif attn_bound == "tensor":
         ach = alg["attn_flops"] / t_attn / 1e12
-        roof = dict(kernel="verify_attention", bound="tensor", achieved=ach, peak=pk["tflops"], unit="TFLOP/s",
-                    frac=ach / pk["tflops"], traffic=NCU_TRAFFIC["verify_attention"].get(cfg.name),
-                    algorithmic_flops=alg["attn_flops"], peak_source=pk["source"])
+        roof = dict(kernel="verify_attention", bound="tensor", achieved=ach, peak=pk["tflops_sustained"], unit="TFLOP/s",
+                    frac=ach / pk["tflops_sustained"], traffic=NCU_TRAFFIC["verify_attention"].get(cfg.name),
+                    algorithmic_flops=alg["attn_flops"], peak_source=pk["source"],
+                    note="timed back to back for 0.25 s, hence against the sustained tensor peak; "
+                         "burst time and burst peak: stages.attention.frac_burst")
     else:
         ach = alg["attn_bytes"] / t_attn / 1e9
         roof = dict(kernel="verify_attention", bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=ach / pk["hbm_gbs"], traffic=NCU_TRAFFIC["verify_attention"].get(cfg.name),
                     algorithmic_bytes=alg["attn_bytes"], peak_source=pk["source"])
+    return dict(value=value, ms_per_step=ms_per_step, steps=steps, clocks=clocks, stages=stages, roofline=roof,
+                e2e=e2e, t=(t_attn, t_topk, t_acc), base_attn=base_attn if full else None,
+                base_vi=base_vi if full else None,
+                launch=("plain launches" if graphs is None else
+                        "cuda graph replay, one graph per step" if round_graph is None else
+                        "cuda graph replay, one graph per round of %d steps" % round_len))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="tsd", choices=["tsd", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the shorter measurements of the other single-GPU workloads")
+    ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graph replay")
+    ap.add_argument("--graph-per-step", action="store_true", help="one graph launch per step instead of one per round of input copies")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "tsd" else args.warmup
+
+    from paper_2608_27514_b200 import workloads as W
+    cfg = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import gc
+    import numpy as np
+    import torch
+    from paper_2608_27514_b200 import binding as B
+    from paper_2608_27514_b200.step import VerifyStep
+
+    from paper_2608_27514_b200 import replicas
+    rank, local_rank, world = replicas.world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    B.lib()  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    replicas.init("nccl", dev)
+    pk = peaks()
+
+    m = measure_workload(cfg, args, torch, np, B, W, VerifyStep, replicas, dev, local_rank, world, pk, full=True)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        cpu = time_oracle_sample(cfg, m["base_attn"], m["base_vi"], 12.0, oracle, np)
+    m["base_attn"] = m["base_vi"] = None
+
+    # the other workloads of the target (every config matches the oracle; attention and the
+    # vocabulary pass against their rooflines), measured the same way with fewer steps
+    per_workload = {}
+    if world == 1 and not args.no_per_workload and args.workload == "cfg2":
+        for name in ("cfg3", "cfg4", "cfg5"):
+            gc.collect()
+            torch.cuda.empty_cache()
+            o = measure_workload(W.CONFIGS[name], args, torch, np, B, W, VerifyStep, replicas, dev, local_rank,
+                                 world, pk, full=False)
+            per_workload[name] = dict(config=base_config(W.CONFIGS[name], world), value=o["value"], unit=UNIT,
+                                      ms_per_step=o["ms_per_step"], steps=o["steps"], clocks=o["clocks"],
+                                      stages=o["stages"], roofline=o["roofline"])
 
     if rank != 0:
         replicas.shutdown()
         return
 
-    cpu = None
-    if world == 1 and not args.no_cpu_baseline:
-        import oracle
-        oracle.build()
-        cpu = time_oracle_sample(cfg, base_attn, base_vi, 20.0, oracle, np)
-
-    launches_per_step = 3  # attention, confidence/top-k, acceptance (the ticket memset is not a kernel of ours)
+    t_attn, t_topk, t_acc = m["t"]
+    launches_per_step = 3  # attention, confidence/top-k, acceptance
     line = dict(
-        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        metric=METRIC, value=m["value"], unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=m["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="bf16" if cfg.dtype == "bf16" else "f32", data="synthetic",
-        config=dict(base_config(cfg, world),
-                    l2_hygiene=("inputs larger than L2" if n_copies == 1 else
-                                "rotating %d input copies (%.0f MB total, L2 is 126 MB)"
-                                % (n_copies, n_copies * in_bytes / 1e6)),
-                    launch=("plain launches" if graphs is None else
-                            "cuda graph replay, one graph per step" if round_graph is None else
-                            "cuda graph replay, one graph per round of %d steps" % round_len)),
-        clocks=clocks,
-        e2e=dict(value=world * cfg.rows / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=int(h2d),
-                 d2h_bytes_per_step=int(d2h), ms_per_step=e2e_ms),
+        config=base_config(cfg, world), launch=m["launch"],
+        clocks=m["clocks"],
+        e2e=dict(value=world * cfg.rows / (m["e2e"]["ms"] * 1e-3), unit=UNIT, h2d_bytes_per_step=m["e2e"]["h2d"],
+                 d2h_bytes_per_step=m["e2e"]["d2h"], ms_per_step=m["e2e"]["ms"]),
         gpu_launches=launches_per_step * args.steps,
-        roofline=roof, stages=stages, cpu_baseline=cpu,
+        roofline=m["roofline"], stages=m["stages"], cpu_baseline=cpu,
         # secondary line: a 32-layer model runs the attention stage once per layer and the vocabulary
         # pass and the acceptance once per step; from the per-stage timings above
         secondary=dict(metric="verified draft-token rows per second with 32 attention layers per step",
                        value=world * cfg.rows / (32 * t_attn + t_topk + t_acc), unit=UNIT,
-                       attention_layers_per_step=32))
+                       attention_layers_per_step=32),
+        per_workload=per_workload)
     print(json.dumps(line))
     replicas.shutdown()
 

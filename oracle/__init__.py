@@ -11,6 +11,7 @@ bookkeeping that turns an accepted path into the next root and its sequential st
 ``fp8`` the e4m3 decode and dequantisation of the FP8 K/V cache variant.
 """
 from .binding import (  # noqa: F401
+    BUILD_FLAGS,
     build,
     num_threads,
     dense_mask,

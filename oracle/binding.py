@@ -12,14 +12,28 @@ _LIB = os.path.join(_HERE, "libtsd_oracle.so")
 _lib = None
 
 
+# -ffp-contract=off keeps every product and sum a separate IEEE operation (no fused multiply-add
+# slipped in by -march=native), so the oracle's bits do not depend on the host's instruction set;
+# nothing is reassociated without -ffast-math.
+BUILD_FLAGS = "-O3 -march=native -ffp-contract=off -fopenmp"
+_FLAGS_FILE = os.path.join(_HERE, "libtsd_oracle.flags")
+
+
 def build(force=False):
-    """Compile the oracle with gcc (-O2, OpenMP over rows)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    """Compile the oracle with gcc (OpenMP over rows); rebuilt when the source or the flags change."""
+    stale = force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if not stale:
+        try:
+            with open(_FLAGS_FILE) as f:
+                stale = f.read().strip() != BUILD_FLAGS
+        except OSError:
+            stale = True
+    if stale:
         tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", _SRC, "-o", tmp, "-lm"]
-        )
+        subprocess.check_call(["gcc"] + BUILD_FLAGS.split() + ["-std=c11", "-fPIC", "-shared", _SRC, "-o", tmp, "-lm"])
         os.replace(tmp, _LIB)
+        with open(_FLAGS_FILE, "w") as f:
+            f.write(BUILD_FLAGS + "\n")
     return _LIB
 
 

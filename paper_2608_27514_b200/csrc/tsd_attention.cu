@@ -2,6 +2,38 @@
 // (bf16, head_dim 128) and the CUDA-core kernel (everything else).
 #include "tsd_common.cuh"
 
+namespace tsd {
+
+// Every host-side check of the attention call, shared by the entry points that end in it: a call
+// that is going to be rejected must be rejected before anything has been launched.
+int check_attention_args(const tsd_layout* L, const void* mask, const void* q, int64_t q_stride_b,
+                         int64_t q_stride_row, int64_t q_stride_head, const void* k_cache, const void* v_cache,
+                         int64_t c_stride_b, int64_t c_stride_row, int64_t c_stride_head, const void* k_draft,
+                         const void* v_draft, int64_t d_stride_b, int64_t d_stride_row, int64_t d_stride_head,
+                         const void* out, int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head,
+                         float sm_scale, const void* workspace) {
+  int rc = validate_layout(L);
+  if (rc != TSD_OK) return rc;
+  if (!mask || !q || !k_draft || !v_draft || !out) return TSD_ERR_INVALID_ARG;
+  if (L->n_cache > 0 && (!k_cache || !v_cache)) return TSD_ERR_INVALID_ARG;
+  if (!(sm_scale == sm_scale)) return TSD_ERR_INVALID_ARG;
+  const void* ptrs[] = {mask, q, k_cache, v_cache, k_draft, v_draft, out, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return TSD_ERR_INVALID_ARG;
+  const int esize = L->dtype == TSD_F32 ? 4 : 2;
+  const int64_t strides[] = {q_stride_b, q_stride_row, q_stride_head, c_stride_b, c_stride_row,
+                             c_stride_head, d_stride_b, d_stride_row, d_stride_head, o_stride_b,
+                             o_stride_row, o_stride_head};
+  for (int64_t st : strides)
+    if (st < 0 || (st * esize) % 16 != 0) return TSD_ERR_INVALID_ARG;
+  if (q_stride_head < L->head_dim || c_stride_head < L->head_dim || d_stride_head < L->head_dim ||
+      o_stride_head < L->head_dim)
+    return TSD_ERR_INVALID_ARG;
+  return TSD_OK;
+}
+
+}  // namespace tsd
+
 extern "C" {
 
 size_t tsd_verify_attention_workspace_bytes(const tsd_layout* L) {
@@ -17,23 +49,11 @@ int tsd_verify_attention(const tsd_layout* L, const void* mask, const void* q, i
                          int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head, float* lse,
                          float sm_scale, void* workspace, size_t workspace_bytes, uint32_t flags,
                          uint32_t* status, tsd_stream_t stream) {
-  int rc = tsd::validate_layout(L);
+  int rc = tsd::check_attention_args(L, mask, q, q_stride_b, q_stride_row, q_stride_head, k_cache, v_cache,
+                                     c_stride_b, c_stride_row, c_stride_head, k_draft, v_draft, d_stride_b,
+                                     d_stride_row, d_stride_head, out, o_stride_b, o_stride_row, o_stride_head,
+                                     sm_scale, workspace);
   if (rc != TSD_OK) return rc;
-  if (!mask || !q || !k_draft || !v_draft || !out) return TSD_ERR_INVALID_ARG;
-  if (L->n_cache > 0 && (!k_cache || !v_cache)) return TSD_ERR_INVALID_ARG;
-  if (!(sm_scale == sm_scale)) return TSD_ERR_INVALID_ARG;
-  const void* ptrs[] = {mask, q, k_cache, v_cache, k_draft, v_draft, out, workspace};
-  for (const void* p : ptrs)
-    if (p && !tsd::aligned16(p)) return TSD_ERR_INVALID_ARG;
-  const int esize = L->dtype == TSD_F32 ? 4 : 2;
-  const int64_t strides[] = {q_stride_b, q_stride_row, q_stride_head, c_stride_b, c_stride_row,
-                             c_stride_head, d_stride_b, d_stride_row, d_stride_head, o_stride_b,
-                             o_stride_row, o_stride_head};
-  for (int64_t st : strides)
-    if (st < 0 || (st * esize) % 16 != 0) return TSD_ERR_INVALID_ARG;
-  if (q_stride_head < L->head_dim || c_stride_head < L->head_dim || d_stride_head < L->head_dim ||
-      o_stride_head < L->head_dim)
-    return TSD_ERR_INVALID_ARG;
 
   tsd::AttnArgs a;
   a.L = *L;

@@ -43,6 +43,12 @@ inline MaskDims mask_dims(const tsd_layout& L) {
 }
 
 int validate_layout(const tsd_layout* L);
+int check_attention_args(const tsd_layout* L, const void* mask, const void* q, int64_t q_stride_b,
+                         int64_t q_stride_row, int64_t q_stride_head, const void* k_cache, const void* v_cache,
+                         int64_t c_stride_b, int64_t c_stride_row, int64_t c_stride_head, const void* k_draft,
+                         const void* v_draft, int64_t d_stride_b, int64_t d_stride_row, int64_t d_stride_head,
+                         const void* out, int64_t o_stride_b, int64_t o_stride_row, int64_t o_stride_head,
+                         float sm_scale, const void* workspace);
 
 // attention launchers (defined in their own translation units)
 struct AttnArgs {

@@ -12,8 +12,8 @@ namespace tsd {
 
 __global__ void __launch_bounds__(256)
 dequant_e4m3_kernel(const uint8_t* __restrict__ src, int64_t ss_b, int64_t ss_r, int64_t ss_h,
-                    const float* __restrict__ scale, __nv_bfloat16* __restrict__ dst, int Nc, int H, int d,
-                    int64_t n_vec) {
+                    const float* __restrict__ scale, const int32_t* __restrict__ mask_blob,
+                    __nv_bfloat16* __restrict__ dst, int Nc, int H, int d, int64_t n_vec) {
   const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // one vector = 16 consecutive codes
   if (v >= n_vec) return;
   const int vec_per_head = d / 16;
@@ -21,6 +21,14 @@ dequant_e4m3_kernel(const uint8_t* __restrict__ src, int64_t ss_b, int64_t ss_r,
   const int h = (int)((v / vec_per_head) % H);
   const int64_t row = (v / vec_per_head / H) % Nc;
   const int64_t s = v / vec_per_head / H / Nc;
+  uint4* o = reinterpret_cast<uint4*>(dst + (((s * Nc + row) * H + h) * (int64_t)d + c * 16));
+  // rows at or past the sequence's cache length (from the mask blob) hold whatever the caller left
+  // there, the NaN codes 0x7f / 0xff included: they are written as zeros and never decoded
+  if (row >= min(max(mask_blob[kHdrWords + s], 0), Nc)) {
+    o[0] = make_uint4(0u, 0u, 0u, 0u);
+    o[1] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
   const uint4 w = *reinterpret_cast<const uint4*>(src + s * ss_b + row * ss_r + h * ss_h + c * 16);
   const float sc = scale ? scale[s * H + h] : 1.f;
   const uint32_t words[4] = {w.x, w.y, w.z, w.w};
@@ -36,7 +44,6 @@ dequant_e4m3_kernel(const uint8_t* __restrict__ src, int64_t ss_b, int64_t ss_r,
       out[2 * i + j] = *reinterpret_cast<const uint32_t*>(&b);
     }
   }
-  uint4* o = reinterpret_cast<uint4*>(dst + (((s * Nc + row) * H + h) * (int64_t)d + c * 16));
   o[0] = make_uint4(out[0], out[1], out[2], out[3]);
   o[1] = make_uint4(out[4], out[5], out[6], out[7]);
 }
@@ -63,10 +70,18 @@ extern "C" int tsd_verify_attention_fp8_cache(
   int rc = tsd::validate_layout(L);
   if (rc != TSD_OK) return rc;
   if (L->dtype != TSD_BF16) return TSD_ERR_UNSUPPORTED;
+  if (L->n_cache > 0 && !workspace) return TSD_ERR_INVALID_ARG;
   if (workspace_bytes < tsd_verify_attention_fp8_cache_workspace_bytes(L)) return TSD_ERR_WORKSPACE;
   const size_t inner = (tsd_verify_attention_workspace_bytes(L) + 255) / 256 * 256;
   const size_t half = tsd::expanded_bytes(*L);
   char* ws = static_cast<char*>(workspace);
+  const int64_t hs = L->head_dim, rs = (int64_t)L->n_kv_heads * hs, bs = (int64_t)L->n_cache * rs;
+  // every check of the attention call that follows, before the first launch: a rejected call launches nothing
+  rc = tsd::check_attention_args(L, mask, q, q_stride_b, q_stride_row, q_stride_head,
+                                 L->n_cache > 0 ? ws + inner : nullptr, L->n_cache > 0 ? ws + inner + half : nullptr,
+                                 bs, rs, hs, k_draft, v_draft, d_stride_b, d_stride_row, d_stride_head, out,
+                                 o_stride_b, o_stride_row, o_stride_head, sm_scale, inner ? workspace : nullptr);
+  if (rc != TSD_OK) return rc;
   if (L->n_cache > 0) {
     if (!k_cache_e4m3 || !v_cache_e4m3 || !workspace || !tsd::aligned16(workspace) || !tsd::aligned16(k_cache_e4m3) ||
         !tsd::aligned16(v_cache_e4m3))
@@ -81,12 +96,11 @@ extern "C" int tsd_verify_attention_fp8_cache(
     for (int t = 0; t < 2; ++t) {
       tsd::dequant_e4m3_kernel<<<blocks, 256, 0, stream>>>(
           static_cast<const uint8_t*>(srcs[t]), c_stride_b, c_stride_row, c_stride_head, scales[t],
-          reinterpret_cast<__nv_bfloat16*>(ws + inner + t * half), L->n_cache, L->n_kv_heads, L->head_dim, n_vec);
+          static_cast<const int32_t*>(mask), reinterpret_cast<__nv_bfloat16*>(ws + inner + t * half), L->n_cache, L->n_kv_heads, L->head_dim, n_vec);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) return tsd::cuda_fail(e, "dequant_e4m3_kernel");
     }
   }
-  const int64_t hs = L->head_dim, rs = (int64_t)L->n_kv_heads * hs, bs = (int64_t)L->n_cache * rs;
   return tsd_verify_attention(L, mask, q, q_stride_b, q_stride_row, q_stride_head,
                               L->n_cache > 0 ? ws + inner : nullptr, L->n_cache > 0 ? ws + inner + half : nullptr, bs, rs,
                               hs, k_draft, v_draft, d_stride_b, d_stride_row, d_stride_head, out, o_stride_b,
