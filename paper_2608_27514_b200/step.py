@@ -23,7 +23,9 @@ class VerifyStep:
         u8 = lambda n: torch.empty(max(int(n), 16), dtype=torch.uint8, device=dev)
         self.mask = u8(B.tsd_branch_mask_bytes(self.layout))
         self.attn_ws = u8(B.tsd_verify_attention_workspace_bytes(self.layout))
-        self.topk_ws = u8(B.tsd_confidence_topk_workspace_bytes(rows, V, k))
+        # zeroed once, as the header asks: the calls keep its ticket words at 0 from then on
+        self.topk_ws = torch.zeros(max(int(B.tsd_confidence_topk_workspace_bytes(rows, V, k)), 16),
+                                   dtype=torch.uint8, device=dev)
         self.out = torch.empty((S, N, Hq, d), dtype=dtype, device=dev)
         self.attn_lse = torch.empty((S, Hq, N), dtype=torch.float32, device=dev)
         self.conf = torch.empty(rows, dtype=torch.float32, device=dev)
