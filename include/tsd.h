@@ -196,7 +196,8 @@ int tsd_selftest_bounded_wait(uint32_t* status, uint32_t poll_limit, tsd_stream_
  *   k_scale, v_scale             device fp32 [batch, n_kv_heads], nullable (= 1);
  *   workspace    tsd_verify_attention_fp8_cache_workspace_bytes() bytes, 16-byte aligned; it is
  *                scratch (can be shared by all layers), the persistent cache stays 8-bit.
- * Only for layout dtype TSD_BF16 (else TSD_ERR_UNSUPPORTED).
+ * Only for layout dtype TSD_BF16, batch <= 65535 and fewer than 2^31 16-code
+ * vectors per sequence and cache (else TSD_ERR_UNSUPPORTED).
  * ------------------------------------------------------------------------- */
 size_t tsd_verify_attention_fp8_cache_workspace_bytes(const tsd_layout* layout);
 int tsd_verify_attention_fp8_cache(const tsd_layout* layout, const void* mask, const void* q,

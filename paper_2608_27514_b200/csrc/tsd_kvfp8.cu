@@ -2,29 +2,34 @@
 // (Section 3.3, App. A); storing it as e4m3 halves its footprint, which is what bounds how many
 // sequences a GPU can hold.  A cached value is bf16(decode_e4m3(code) * scale[sequence, kv head])
 // (the product and the rounding in fp32 -> bf16).  The cache is expanded into the caller's
-// workspace by a streaming kernel (16 codes in, 32 bytes out per thread) and the attention kernels
-// then run unchanged on the expanded copy; the workspace is transient and can be shared by all
-// layers, the persistent cache stays 8-bit.
+// workspace by one streaming launch for both caches (16 codes in, 32 bytes out per thread; grid
+// y = sequence, z = K or V, so that the indices stay 32-bit) and the attention kernels then run
+// unchanged on the expanded copy; the workspace is transient and can be shared by all layers, the
+// persistent cache stays 8-bit.
 #include <cuda_fp8.h>
 #include "tsd_common.cuh"
 
 namespace tsd {
 
 __global__ void __launch_bounds__(256)
-dequant_e4m3_kernel(const uint8_t* __restrict__ src, int64_t ss_b, int64_t ss_r, int64_t ss_h,
-                    const float* __restrict__ scale, const int32_t* __restrict__ mask_blob,
-                    __nv_bfloat16* __restrict__ dst, int Nc, int H, int d, int64_t n_vec) {
-  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;  // one vector = 16 consecutive codes
-  if (v >= n_vec) return;
-  const int vec_per_head = d / 16;
-  const int c = (int)(v % vec_per_head);
-  const int h = (int)((v / vec_per_head) % H);
-  const int64_t row = (v / vec_per_head / H) % Nc;
-  const int64_t s = v / vec_per_head / H / Nc;
+dequant_e4m3_kernel(const uint8_t* __restrict__ k_src, const uint8_t* __restrict__ v_src, int64_t ss_b, int64_t ss_r,
+                    int64_t ss_h, const float* __restrict__ k_scale, const float* __restrict__ v_scale,
+                    const int32_t* __restrict__ mask_blob, __nv_bfloat16* __restrict__ k_dst,
+                    __nv_bfloat16* __restrict__ v_dst, int Nc, int H, int d, uint32_t vec_per_seq) {
+  const uint32_t v = blockIdx.x * blockDim.x + threadIdx.x;  // one vector = 16 consecutive codes of sequence s
+  if (v >= vec_per_seq) return;
+  const uint32_t vec_per_head = (uint32_t)d / 16u, vec_per_row = vec_per_head * (uint32_t)H;
+  const uint32_t row = v / vec_per_row, cv = v - row * vec_per_row;
+  const uint32_t h = cv / vec_per_head, c = cv - h * vec_per_head;
+  const int64_t s = blockIdx.y;
+  const bool is_v = blockIdx.z != 0;
+  const uint8_t* src = is_v ? v_src : k_src;
+  const float* scale = is_v ? v_scale : k_scale;
+  __nv_bfloat16* dst = is_v ? v_dst : k_dst;
   uint4* o = reinterpret_cast<uint4*>(dst + (((s * Nc + row) * H + h) * (int64_t)d + c * 16));
   // rows at or past the sequence's cache length (from the mask blob) hold whatever the caller left
   // there, the NaN codes 0x7f / 0xff included: they are written as zeros and never decoded
-  if (row >= min(max(mask_blob[kHdrWords + s], 0), Nc)) {
+  if ((int)row >= min(max(mask_blob[kHdrWords + s], 0), Nc)) {
     o[0] = make_uint4(0u, 0u, 0u, 0u);
     o[1] = make_uint4(0u, 0u, 0u, 0u);
     return;
@@ -89,17 +94,16 @@ extern "C" int tsd_verify_attention_fp8_cache(
     if (c_stride_b < 0 || c_stride_row < 0 || c_stride_head < L->head_dim || c_stride_b % 16 || c_stride_row % 16 ||
         c_stride_head % 16)
       return TSD_ERR_INVALID_ARG;
-    const int64_t n_vec = (int64_t)L->batch * L->n_cache * L->n_kv_heads * (L->head_dim / 16);
-    const unsigned blocks = (unsigned)((n_vec + 255) / 256);
-    const void* srcs[2] = {k_cache_e4m3, v_cache_e4m3};
-    const float* scales[2] = {k_scale, v_scale};
-    for (int t = 0; t < 2; ++t) {
-      tsd::dequant_e4m3_kernel<<<blocks, 256, 0, stream>>>(
-          static_cast<const uint8_t*>(srcs[t]), c_stride_b, c_stride_row, c_stride_head, scales[t],
-          static_cast<const int32_t*>(mask), reinterpret_cast<__nv_bfloat16*>(ws + inner + t * half), L->n_cache, L->n_kv_heads, L->head_dim, n_vec);
-      cudaError_t e = cudaGetLastError();
-      if (e != cudaSuccess) return tsd::cuda_fail(e, "dequant_e4m3_kernel");
-    }
+    const int64_t vec_per_seq = (int64_t)L->n_cache * L->n_kv_heads * (L->head_dim / 16);
+    if (vec_per_seq > 0x7fffff00ll || L->batch > 65535) return TSD_ERR_UNSUPPORTED;  // 32-bit indices, grid y
+    const dim3 grid((unsigned)((vec_per_seq + 255) / 256), (unsigned)L->batch, 2);
+    tsd::dequant_e4m3_kernel<<<grid, 256, 0, stream>>>(
+        k_cache_e4m3, v_cache_e4m3, c_stride_b, c_stride_row, c_stride_head, k_scale, v_scale,
+        static_cast<const int32_t*>(mask), reinterpret_cast<__nv_bfloat16*>(ws + inner),
+        reinterpret_cast<__nv_bfloat16*>(ws + inner + half), L->n_cache, L->n_kv_heads, L->head_dim,
+        (uint32_t)vec_per_seq);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return tsd::cuda_fail(e, "dequant_e4m3_kernel");
   }
   return tsd_verify_attention(L, mask, q, q_stride_b, q_stride_row, q_stride_head,
                               L->n_cache > 0 ? ws + inner : nullptr, L->n_cache > 0 ? ws + inner + half : nullptr, bs, rs,
