@@ -158,6 +158,10 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
   asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
@@ -429,6 +433,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) TSD_TR_ALWAYS(0, 200);
+  // The copy engine fetches a tensor map from global memory the first time a copy names it, and the
+  // issuing thread waits for that (measured: the first K request left 1.8 k clocks after the producer
+  // reached it).  Ask for all six at once, now.
+  if (tid == kVProducerWarp * 32) {
+    prefetch_tensormap(&map_q);
+    prefetch_tensormap(&map_kc);
+    prefetch_tensormap(&map_vc);
+    prefetch_tensormap(&map_kd);
+    prefetch_tensormap(&map_vd);
+    prefetch_tensormap(&map_o);
+  }
   const int32_t* mask = p.mask;
   const int n_my = (int)blockIdx.x < p.n_items ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   // item -> (sequence, query head, query tile); query tiles of a head, then heads, then sequences
@@ -453,6 +468,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     item_T[it] = n_ct + 2 * n_dt;
   }
 
+  // Coordinates of the block's first item for the two producer lanes: worked out here, while the
+  // block is still setting up, so that their first requests after the sync are a few instructions.
+  int s_first = 0, g_first = 0;
+  if (lane == 0 && (warp == kKProducerWarp || warp == kVProducerWarp) && n_my > 0) {
+    int h, qt;
+    item_coords(0, s_first, h, qt);
+    g_first = h / p.group;
+  }
   if (warp == kKProducerWarp && lane == 0) {
     abort_flag[0] = 0;
     abort_flag[1] = 0;  // scratch flag for the drain waits
@@ -534,6 +557,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int n_stage = is_k ? kNK : kNV;
       int G = 0, b = 0;       // tile count, its stage = G mod n_stage
       uint32_t ph = 0;        // phase of that stage's barriers = (G / n_stage) & 1
+      // The first cached tiles of the first item, one per stage, go out before the general loop
+      // below is entered: on its first pass that loop costs ~1.5 k clocks of instruction fetches and
+      // single-lane index arithmetic before its first request (measured), and the whole block
+      // waits for these tiles.
+      const int n_pre = n_run > 0 ? min(n_stage, (item_clen[0] + kKeys - 1) / kKeys) : 0;
+      for (int t = 0; t < n_pre; ++t) {
+        const uint32_t dst = stage0 + t * kKVBytes, full_bar = bar(full0 + t);
+        mbar_expect_tx(full_bar, kKVBytes);
+        if (is_k && t < kNSb) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], 4;" ::"r"(full_bar) : "memory");
+        tma_load_4d(dst, mc, full_bar, 0, g_first, t * kKeys, s_first);
+        tma_load_4d(dst + kSubKV, mc, full_bar, 64, g_first, t * kKeys, s_first);
+      }
+      issued = n_pre;
       for (int it = 0; it < n_run && ok; ++it) {
         // Q of this item must be on its way before its K tiles queue behind it
         while (is_k && ok && q_issued <= it) issue_q(true);
@@ -547,17 +583,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           // the stage is free once the MMAs that read its previous tile have completed
           if (G >= n_stage) ok = mbar_wait(bar(free0 + b), ph ^ 1u, abort_flag, 100);
           if (!ok) break;
-          const bool cached = j < n_ct;
-          const int e = j - n_ct;  // draft key tile e = half (e & 1) of the listed 128-row tile e >> 1
-          const int row = cached ? j * kKeys : rec[2 + 2 * (e >> 1)] * kTile + (e & 1) * kKeys;
-          const CUtensorMap* m = cached ? mc : md;
-          const uint32_t dst = stage0 + b * kKVBytes, full_bar = bar(full0 + b);
-          mbar_expect_tx(full_bar, kKVBytes);
-          // no softmax has run before the first three tiles: their S buffers are free from the start
-          if (is_k && G < kNSb) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], 4;" ::"r"(full_bar) : "memory");
-          tma_load_4d(dst, m, full_bar, 0, g, row, s);
-          tma_load_4d(dst + kSubKV, m, full_bar, 64, g, row, s);
-          issued = G + 1;
+          if (G >= n_pre) {
+            const bool cached = j < n_ct;
+            const int e = j - n_ct;  // draft key tile e = half (e & 1) of the listed 128-row tile e >> 1
+            const int row = cached ? j * kKeys : rec[2 + 2 * (e >> 1)] * kTile + (e & 1) * kKeys;
+            const CUtensorMap* m = cached ? mc : md;
+            const uint32_t dst = stage0 + b * kKVBytes, full_bar = bar(full0 + b);
+            mbar_expect_tx(full_bar, kKVBytes);
+            // no softmax has run before the first three tiles: their S buffers are free from the start
+            if (is_k && G < kNSb) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], 4;" ::"r"(full_bar) : "memory");
+            tma_load_4d(dst, m, full_bar, 0, g, row, s);
+            tma_load_4d(dst + kSubKV, m, full_bar, 64, g, row, s);
+            issued = G + 1;
+          }
           TSD_TR(is_k ? 0 : 1, G);
           if (++b == n_stage) { b = 0; ph ^= 1u; }
         }
